@@ -1,0 +1,162 @@
+/*
+ * specverify.h -- C ABI of libspecverify: batched verification of a draft token tree on one GPU.
+ *
+ * The library implements the verification step of multi-path speculative decoding (paper
+ * Section 2, step 3): given target and draft logits on the nodes of a draft tree, the tree, the
+ * sampling parameters and caller-supplied uniforms, it selects one accepted node and one
+ * correction ("bonus") token so that the emitted tokens follow the target distribution.
+ *
+ * General rules for every entry point
+ *   - `extern "C"`, plain pointers and sizes.  Unless a parameter says "host", a data pointer is
+ *     a DEVICE pointer owned by the caller; the library only borrows it until the work it
+ *     enqueued on `stream` has finished.  `SpecIn` / `SpecOut` themselves are host structs, read
+ *     during the call only.
+ *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = the legacy default stream).  Calls
+ *     enqueue kernels and return; they never synchronise, allocate or free.
+ *   - Scratch memory comes from the caller: `ws` (device, 256-byte aligned) of at least
+ *     `spec_workspace_bytes()` bytes.  Two calls that may overlap on the GPU need two workspaces.
+ *   - Return value: SPEC_OK or a negative SPEC_ERR_* found on the host before anything was
+ *     enqueued.  Problems only visible on the device (bad topology or token, a non-finite row, a
+ *     bounded wait that ran out) are reported per sequence in `SpecOut.status` (a SPEC_DEV_*
+ *     code); that sequence gets accept_len = -1 and accepted_node = -1.  Nothing traps.
+ *   - There is no CPU fallback.
+ *
+ * Tree layout (Definition 3.1, Definition 5.2): node 0 is the root (the current context);
+ * parent[0] = -1 and parent[i] < i.  The child list of a node is the set of nodes naming it as
+ * parent, in increasing index order; that is the order in which children are tried.  Equal tokens
+ * under one parent stay separate nodes (multiplicity, Section 3.2).  At most SPEC_MAX_CHILDREN
+ * children per node and SPEC_MAX_NODES nodes per sequence.
+ *
+ * Sampling distribution of a row (Section 4 names temperature and nucleus sampling; top-k is an
+ * addition): y = z / T, softmax; top-k keeps every token whose logit is >= the k-th largest logit
+ * value; top-p then keeps the fewest leading groups of equal-logit tokens whose mass (within the
+ * top-k set) reaches top_p; renormalise.  The same transform is applied to target and draft rows.
+ */
+#ifndef SPECVERIFY_H
+#define SPECVERIFY_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPEC_MAX_CHILDREN 16
+#define SPEC_MAX_NODES 1024
+
+/* host-side return codes */
+#define SPEC_OK 0
+#define SPEC_ERR_NULL (-1)        /* a required pointer is NULL                                  */
+#define SPEC_ERR_SHAPE (-2)       /* B, N, V or a stride is out of range                         */
+#define SPEC_ERR_DTYPE (-3)       /* logits_dtype is neither SPEC_F32 nor SPEC_BF16              */
+#define SPEC_ERR_PARAM (-4)       /* temperature <= 0 or not finite, top_p outside (0,1], top_k < 0 */
+#define SPEC_ERR_WORKSPACE (-5)   /* ws NULL, misaligned or too small                            */
+#define SPEC_ERR_UNSUPPORTED (-6) /* vocabulary too large for the on-chip plan of this device    */
+#define SPEC_ERR_CUDA (-7)        /* a CUDA runtime call failed (launch configuration, no device) */
+
+/* per-sequence device status codes (SpecOut.status) */
+#define SPEC_DEV_OK 0
+#define SPEC_DEV_TOPOLOGY 1       /* parent[0] != -1, parent[i] outside [0,i), too many children */
+#define SPEC_DEV_TOKEN 2          /* token outside [0,V)                                         */
+#define SPEC_DEV_NONFINITE 3      /* a logit row holds NaN / +inf, or only -inf                  */
+#define SPEC_DEV_TIMEOUT 4        /* a bounded on-device wait ran out                            */
+
+#define SPEC_F32 0
+#define SPEC_BF16 1
+
+typedef struct {
+    int32_t B, N, V;              /* sequences, nodes per sequence (root included), vocabulary   */
+    int32_t logits_dtype;         /* SPEC_F32 or SPEC_BF16                                        */
+    const void *target_logits;    /* [B,N,V] row of node a of sequence b at b*seq_stride + a*node_stride */
+    const void *draft_logits;     /* same layout; rows of nodes without children are never read  */
+    int64_t seq_stride;           /* in elements                                                  */
+    int64_t node_stride;          /* in elements, >= V; the V entries of a row are contiguous     */
+    const int32_t *parent;        /* [N], or [B,N] with topo_seq_stride = N                       */
+    int64_t topo_seq_stride;      /* 0: one topology shared by the batch                          */
+    const int32_t *token;         /* [B,N] draft token of each node; token[b,0] is ignored        */
+    float temperature;            /* > 0                                                          */
+    int32_t top_k;                /* 0 = off                                                      */
+    float top_p;                  /* in (0,1]; 1 = off                                            */
+    const float *temperature_per_seq; /* optional [B]; overrides `temperature` when not NULL      */
+    const float *u_accept;        /* [B,N] uniforms in [0,1): entry of node a decides a's test    */
+    const float *u_bonus;         /* [B,N] uniforms in [0,1): the stop node's entry draws the bonus */
+} SpecIn;
+
+typedef struct {
+    int32_t *accepted_node;       /* [B] index of the accepted node (0 = nothing accepted)        */
+    int32_t *accept_len;          /* [B] tau = depth of the accepted node                          */
+    int32_t *out_tokens;          /* [B,N] tokens on the accepted path, then the bonus, then -1   */
+    int32_t *bonus_token;         /* [B]                                                           */
+    int32_t *status;              /* [B] SPEC_DEV_*                                                */
+    /* optional outputs: skipped when NULL */
+    float *residual;              /* [B,V] the distribution the bonus token was drawn from         */
+    float *node_thr;              /* [B,N] threshold node a is tested with as if it were reached:
+                                     SpecInfer: min(1, P/q) after its earlier siblings were rejected
+                                     (asking for it disables the early exit after an accepted
+                                     sibling); Traversal: the final weight of a.  Root: 1          */
+    float *node_w_in;             /* [B,N] Traversal only: weight handed to a by its parent        */
+    float *node_features;         /* [B,N,4] entropy (nats) of the target and draft sampling
+                                     distributions and their largest probability:
+                                     H_p, H_q, top1_p, top1_q (q entries 0 for childless nodes)   */
+    float *margin;                /* [B,N+1] |u_accept - threshold| per node (NaN where the node
+                                     was not evaluated), last entry: distance of the bonus draw to
+                                     the nearer CDF boundary, as a fraction of the total mass      */
+} SpecOut;
+
+/* Bytes of scratch the calls below need for these shapes (depends on B, N only).
+ * host pointers.  Returns SPEC_OK or SPEC_ERR_NULL / SPEC_ERR_SHAPE. */
+int32_t spec_workspace_bytes(const SpecIn *in, int64_t *bytes);
+
+/*
+ * Sampling distribution of every node's target (which = 0) or draft (which = 1) row, written to
+ * HBM (Section 4: temperature / nucleus; tie rules above).
+ *   probs      [B,N,V] float, contiguous.  May be NULL when only the statistics are wanted.
+ *   row_stats  optional [B,N,6] float: max of z/T, sum of kept exp(z/T - max), kept count,
+ *              entropy (nats), largest probability, smallest kept logit value.
+ * Only B, N, V, dtype, the logits of the chosen side, strides and the sampling parameters of `in`
+ * are read.  Rows that are not finite produce NaN statistics and zero probabilities.
+ */
+int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats,
+                        void *ws, int64_t ws_bytes, void *stream);
+
+/*
+ * SpecInfer verification (Algorithm 4 used top-down, Section 3.2 "OT-based algorithms"):
+ * starting at the root, try the children of the current node in list order; child x is accepted
+ * when u_accept < min(1, P(x)/q(x)), where P is the node's target distribution after the residual
+ * updates P <- norm((P - q)+) of the siblings rejected before it; on acceptance move to that
+ * child, otherwise stop and draw the bonus token from P by inverse CDF with the node's u_bonus
+ * (from the unmodified target distribution at a childless node).
+ * Fused: logits in, decisions out; no [B,N,V] tensor is written.
+ */
+int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes,
+                              void *stream);
+
+/*
+ * Traversal Verification (Section 3.2, bottom-up; block verification of Section 3.1 on one
+ * path).  Weights flow down: a child with token x gets min(1, w P(x)/q(x)) from its parent's
+ * current (w, P); a node is tested (u_accept < w) only after all its child subtrees were
+ * rejected, each rejection updating the parent to S = sum (wP - q)+, w <- S / (S + 1 - w),
+ * P <- (wP - q)+ / S.  The first node accepted in depth-first post-order wins; the root always
+ * accepts.  The bonus token is drawn from the accepted node's final P with its u_bonus.
+ */
+int32_t spec_verify_traversal(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes,
+                              void *stream);
+
+/*
+ * Inverse-CDF draw (the "Sample Y ~ p" steps of Algorithms 1-4) from R rows of non-negative
+ * weights that need not be normalised: token[r] = smallest t with w_0 + ... + w_t > u[r] * sum(w).
+ *   weights [R,V] float contiguous, u [R] in [0,1), token [R] (-1 for an all-zero row),
+ *   margin optional [R]: distance to the nearer CDF boundary as a fraction of the total.
+ */
+int32_t spec_sample_bonus(const float *weights, int32_t R, int32_t V, const float *u,
+                          int32_t *token, float *margin, void *ws, int64_t ws_bytes, void *stream);
+
+/* Launch plan chosen for a vocabulary size and dtype (host-only query, for benchmarks and tests):
+ * CTAs per cluster, tokens per CTA slice, dynamic shared memory bytes per CTA, threads per CTA. */
+int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, int32_t *slice_len,
+                        int32_t *smem_bytes, int32_t *threads);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECVERIFY_H */

@@ -1,0 +1,323 @@
+"""Thin ctypes binding of libspecverify.so: argument marshalling only.
+
+Every step of the verification path runs inside the CUDA library; this module turns torch tensors
+into the plain pointers of the C ABI (``include/specverify.h``), owns the scratch workspace and
+allocates output tensors.  There is no CPU fallback: a missing library or a missing CUDA device
+raises ``RuntimeError``.
+
+Device-resident API (inputs already in HBM, nothing is synchronised):
+    verify_specinfer / verify_traversal / tree_probs / sample_bonus
+Host API (pinned host buffers in, host results out; copies and one stream sync inside):
+    HostVerifier
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspecverify.so")
+
+SPEC_F32, SPEC_BF16 = 0, 1
+ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_DTYPE",
+          -4: "SPEC_ERR_PARAM", -5: "SPEC_ERR_WORKSPACE", -6: "SPEC_ERR_UNSUPPORTED", -7: "SPEC_ERR_CUDA"}
+EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
+           "spec_sample_bonus", "spec_query_plan")
+
+
+class SpecIn(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("N", C.c_int32), ("V", C.c_int32), ("logits_dtype", C.c_int32),
+        ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+        ("seq_stride", C.c_int64), ("node_stride", C.c_int64),
+        ("parent", C.c_void_p), ("topo_seq_stride", C.c_int64), ("token", C.c_void_p),
+        ("temperature", C.c_float), ("top_k", C.c_int32), ("top_p", C.c_float),
+        ("temperature_per_seq", C.c_void_p), ("u_accept", C.c_void_p), ("u_bonus", C.c_void_p),
+    ]
+
+
+class SpecOut(C.Structure):
+    _fields_ = [
+        ("accepted_node", C.c_void_p), ("accept_len", C.c_void_p), ("out_tokens", C.c_void_p),
+        ("bonus_token", C.c_void_p), ("status", C.c_void_p), ("residual", C.c_void_p),
+        ("node_thr", C.c_void_p), ("node_w_in", C.c_void_p), ("node_features", C.c_void_p),
+        ("margin", C.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH):
+    """dlopen the CUDA library (no device needed for this step) and declare the prototypes."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2602_16994_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(path)
+    lib.spec_workspace_bytes.restype = C.c_int32
+    lib.spec_workspace_bytes.argtypes = [C.POINTER(SpecIn), C.POINTER(C.c_int64)]
+    lib.spec_tree_probs.restype = C.c_int32
+    lib.spec_tree_probs.argtypes = [C.POINTER(SpecIn), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                    C.c_int64, C.c_void_p]
+    for name in ("spec_verify_specinfer", "spec_verify_traversal"):
+        f = getattr(lib, name)
+        f.restype = C.c_int32
+        f.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_void_p, C.c_int64, C.c_void_p]
+    lib.spec_sample_bonus.restype = C.c_int32
+    lib.spec_sample_bonus.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_int64, C.c_void_p]
+    lib.spec_query_plan.restype = C.c_int32
+    lib.spec_query_plan.argtypes = [C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 4
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed: {ERRORS.get(rc, rc)}")
+
+
+def _require_cuda(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise RuntimeError(f"{name} must live on a CUDA device (there is no CPU path)")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def query_plan(V: int, dtype: int = SPEC_BF16) -> dict:
+    lib = load_library()
+    c, sl, sm, nt = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    _check(lib.spec_query_plan(V, dtype, C.byref(c), C.byref(sl), C.byref(sm), C.byref(nt)), "spec_query_plan")
+    return dict(cluster_size=c.value, slice_len=sl.value, smem_bytes=sm.value, threads=nt.value)
+
+
+def make_spec_in(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0,
+                 top_k=0, top_p=1.0, temperature_per_seq=None) -> SpecIn:
+    """Marshal tensors into a SpecIn.  Logits: [B,N,V] float32 or bfloat16, last dim contiguous."""
+    for name, t in (("target_logits", target_logits), ("draft_logits", draft_logits), ("parent", parent),
+                    ("token", token), ("u_accept", u_accept), ("u_bonus", u_bonus)):
+        _require_cuda(t, name)
+    if target_logits.dtype not in (torch.float32, torch.bfloat16) or draft_logits.dtype != target_logits.dtype:
+        raise RuntimeError("logits must both be float32 or both bfloat16")
+    if target_logits.dim() != 3 or target_logits.stride(2) != 1 or draft_logits.stride() != target_logits.stride():
+        raise RuntimeError("logits must be [B,N,V] with a contiguous vocabulary axis and equal strides")
+    B, N, V = target_logits.shape
+    for name, t, dt in (("parent", parent, torch.int32), ("token", token, torch.int32),
+                        ("u_accept", u_accept, torch.float32), ("u_bonus", u_bonus, torch.float32)):
+        if t.dtype != dt or not t.is_contiguous():
+            raise RuntimeError(f"{name} must be a contiguous {dt} tensor")
+    if tuple(token.shape) != (B, N) or tuple(u_accept.shape) != (B, N) or tuple(u_bonus.shape) != (B, N):
+        raise RuntimeError("token, u_accept and u_bonus must be [B,N]")
+    if tuple(parent.shape) not in ((N,), (B, N)):
+        raise RuntimeError("parent must be [N] or [B,N]")
+    return SpecIn(B, N, V, SPEC_F32 if target_logits.dtype == torch.float32 else SPEC_BF16,
+                  _ptr(target_logits), _ptr(draft_logits), target_logits.stride(0), target_logits.stride(1),
+                  _ptr(parent), 0 if parent.dim() == 1 else N, _ptr(token), float(temperature), int(top_k),
+                  float(top_p), _ptr(temperature_per_seq), _ptr(u_accept), _ptr(u_bonus))
+
+
+def workspace_bytes(spec_in: SpecIn) -> int:
+    n = C.c_int64()
+    _check(load_library().spec_workspace_bytes(C.byref(spec_in), C.byref(n)), "spec_workspace_bytes")
+    return int(n.value)
+
+
+@dataclass
+class VerifyOutputs:
+    accepted_node: torch.Tensor
+    accept_len: torch.Tensor
+    out_tokens: torch.Tensor
+    bonus_token: torch.Tensor
+    status: torch.Tensor
+    residual: torch.Tensor | None = None
+    node_thr: torch.Tensor | None = None
+    node_w_in: torch.Tensor | None = None
+    node_features: torch.Tensor | None = None
+    margin: torch.Tensor | None = None
+
+    def as_struct(self) -> SpecOut:
+        return SpecOut(_ptr(self.accepted_node), _ptr(self.accept_len), _ptr(self.out_tokens),
+                       _ptr(self.bonus_token), _ptr(self.status), _ptr(self.residual), _ptr(self.node_thr),
+                       _ptr(self.node_w_in), _ptr(self.node_features), _ptr(self.margin))
+
+
+def alloc_outputs(B, N, V, device, residual=False, node_thr=False, node_w_in=False, features=False,
+                  margin=False) -> VerifyOutputs:
+    i32 = dict(dtype=torch.int32, device=device)
+    f32 = dict(dtype=torch.float32, device=device)
+    return VerifyOutputs(
+        torch.empty(B, **i32), torch.empty(B, **i32), torch.empty((B, N), **i32), torch.empty(B, **i32),
+        torch.empty(B, **i32),
+        torch.empty((B, V), **f32) if residual else None,
+        torch.empty((B, N), **f32) if node_thr else None,
+        torch.empty((B, N), **f32) if node_w_in else None,
+        torch.empty((B, N, 4), **f32) if features else None,
+        torch.empty((B, N + 1), **f32) if margin else None)
+
+
+class Workspace:
+    """Scratch memory for the verify calls; grows on demand, one per stream of concurrent calls."""
+
+    def __init__(self, device):
+        self.device = device
+        self.buf = None
+
+    def get(self, nbytes: int):
+        if self.buf is None or self.buf.numel() < nbytes + 256:
+            self.buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.buf.data_ptr()
+        off = (-base) % 256
+        return C.c_void_p(base + off), self.buf.numel() - off
+
+
+_default_ws = {}
+
+
+def _ws_for(device) -> Workspace:
+    key = str(device)
+    if key not in _default_ws:
+        _default_ws[key] = Workspace(device)
+    return _default_ws[key]
+
+
+def _verify(fn_name, batch_or_in, outputs, workspace, stream, **alloc):
+    lib = load_library()
+    if not torch.cuda.is_available():
+        raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
+    spec_in, keep = batch_or_in
+    B, N, V = spec_in.B, spec_in.N, spec_in.V
+    device = keep[0].device
+    if outputs is None:
+        outputs = alloc_outputs(B, N, V, device, **alloc)
+    ws = workspace or _ws_for(device)
+    ptr, size = ws.get(workspace_bytes(spec_in))
+    so = outputs.as_struct()
+    _check(getattr(lib, fn_name)(C.byref(spec_in), C.byref(so), ptr, size, _stream_ptr(stream)), fn_name)
+    return outputs
+
+
+def _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+             temperature_per_seq):
+    si = make_spec_in(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k,
+                      top_p, temperature_per_seq)
+    return si, (target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature_per_seq)
+
+
+def verify_specinfer(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0,
+                     top_k=0, top_p=1.0, temperature_per_seq=None, outputs=None, workspace=None,
+                     stream=None, residual=False, node_thr=False, features=False, margin=False):
+    """SpecInfer verification of a batch of draft trees (enqueued on the stream; returns device tensors)."""
+    m = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+                 temperature_per_seq)
+    return _verify("spec_verify_specinfer", m, outputs, workspace, stream, residual=residual,
+                   node_thr=node_thr, features=features, margin=margin)
+
+
+def verify_traversal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0,
+                     top_k=0, top_p=1.0, temperature_per_seq=None, outputs=None, workspace=None,
+                     stream=None, residual=False, node_thr=False, node_w_in=False, features=False,
+                     margin=False):
+    """Traversal Verification of a batch of draft trees."""
+    m = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+                 temperature_per_seq)
+    return _verify("spec_verify_traversal", m, outputs, workspace, stream, residual=residual,
+                   node_thr=node_thr, node_w_in=node_w_in, features=features, margin=margin)
+
+
+def tree_probs(logits, which=0, temperature=1.0, top_k=0, top_p=1.0, temperature_per_seq=None,
+               want_probs=True, want_stats=True, stream=None):
+    """Sampling distribution of every row of ``logits`` [B,N,V].  Returns (probs or None, stats or None)."""
+    lib = load_library()
+    _require_cuda(logits, "logits")
+    if logits.dim() != 3 or logits.stride(2) != 1 or logits.dtype not in (torch.float32, torch.bfloat16):
+        raise RuntimeError("logits must be [B,N,V] float32 / bfloat16 with a contiguous vocabulary axis")
+    B, N, V = logits.shape
+    si = SpecIn(B, N, V, SPEC_F32 if logits.dtype == torch.float32 else SPEC_BF16,
+                _ptr(logits), _ptr(logits), logits.stride(0), logits.stride(1), None, 0, None,
+                float(temperature), int(top_k), float(top_p), _ptr(temperature_per_seq), None, None)
+    probs = torch.empty((B, N, V), dtype=torch.float32, device=logits.device) if want_probs else None
+    stats = torch.empty((B, N, 6), dtype=torch.float32, device=logits.device) if want_stats else None
+    _check(lib.spec_tree_probs(C.byref(si), int(which), _ptr(probs), _ptr(stats), None, 0, _stream_ptr(stream)),
+           "spec_tree_probs")
+    return probs, stats
+
+
+def sample_bonus(weights, u, want_margin=False, stream=None):
+    """Inverse-CDF draw from each row of ``weights`` [R,V] float32 with uniforms ``u`` [R]."""
+    lib = load_library()
+    _require_cuda(weights, "weights")
+    _require_cuda(u, "u")
+    if weights.dtype != torch.float32 or not weights.is_contiguous() or weights.dim() != 2:
+        raise RuntimeError("weights must be a contiguous [R,V] float32 tensor")
+    if u.dtype != torch.float32 or not u.is_contiguous() or u.numel() != weights.shape[0]:
+        raise RuntimeError("u must be a contiguous float32 tensor with one entry per row")
+    R, V = weights.shape
+    token = torch.empty(R, dtype=torch.int32, device=weights.device)
+    margin = torch.empty(R, dtype=torch.float32, device=weights.device) if want_margin else None
+    _check(lib.spec_sample_bonus(_ptr(weights), R, V, _ptr(u), _ptr(token), _ptr(margin), None, 0,
+                                 _stream_ptr(stream)), "spec_sample_bonus")
+    return (token, margin) if want_margin else token
+
+
+class HostVerifier:
+    """End-to-end call for callers whose logits live in (pinned) host memory.
+
+    Owns device staging buffers for one batch shape.  ``run`` copies the inputs host->device, enqueues
+    the verifier, copies the decisions device->host and synchronises the stream once.
+    """
+
+    def __init__(self, B, N, V, logits_dtype=torch.bfloat16, device="cuda", algorithm="specinfer"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
+        load_library()
+        self.device = torch.device(device)
+        self.algorithm = algorithm
+        self.shape = (B, N, V)
+        d = self.device
+        self.zp = torch.empty((B, N, V), dtype=logits_dtype, device=d)
+        self.zq = torch.empty((B, N, V), dtype=logits_dtype, device=d)
+        self.parent = torch.empty(N, dtype=torch.int32, device=d)
+        self.token = torch.empty((B, N), dtype=torch.int32, device=d)
+        self.ua = torch.empty((B, N), dtype=torch.float32, device=d)
+        self.ub = torch.empty((B, N), dtype=torch.float32, device=d)
+        self.out = alloc_outputs(B, N, V, d)
+        self.host_out = {k: torch.empty_like(getattr(self.out, k), device="cpu").pin_memory()
+                         for k in ("accepted_node", "accept_len", "out_tokens", "bonus_token", "status")}
+        self.ws = Workspace(d)
+        self.stream = torch.cuda.Stream(device=d)
+
+    def h2d_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.zp, self.zq, self.parent, self.token, self.ua, self.ub))
+
+    def d2h_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in self.host_out.values())
+
+    def run(self, target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0, top_k=0,
+            top_p=1.0):
+        with torch.cuda.stream(self.stream):
+            self.zp.copy_(target_logits, non_blocking=True)
+            self.zq.copy_(draft_logits, non_blocking=True)
+            self.parent.copy_(parent, non_blocking=True)
+            self.token.copy_(token, non_blocking=True)
+            self.ua.copy_(u_accept, non_blocking=True)
+            self.ub.copy_(u_bonus, non_blocking=True)
+            fn = verify_specinfer if self.algorithm == "specinfer" else verify_traversal
+            fn(self.zp, self.zq, self.parent, self.token, self.ua, self.ub, temperature, top_k, top_p,
+               outputs=self.out, workspace=self.ws, stream=self.stream)
+            for k, h in self.host_out.items():
+                h.copy_(getattr(self.out, k), non_blocking=True)
+        self.stream.synchronize()
+        return self.host_out
