@@ -151,6 +151,20 @@ int32_t spec_verify_traversal(const SpecIn *in, const SpecOut *out, void *ws, in
 int32_t spec_sample_bonus(const float *weights, int32_t R, int32_t V, const float *u,
                           int32_t *token, float *margin, void *ws, int64_t ws_bytes, void *stream);
 
+/*
+ * Host-buffer form of the two verifiers (the verification step of Section 2 for a caller whose
+ * logits sit in host memory).  Every data pointer of `in` and `out` is a HOST pointer (pinned
+ * memory gives asynchronous copies); logits must be dense ([B,N,V] contiguous).  `dev_buf` is a
+ * DEVICE buffer of at least spec_host_staging_bytes() bytes, 256-byte aligned, owned by the
+ * caller; inputs are copied into it, the verifier (algorithm 0 = SpecInfer, 1 = Traversal) runs
+ * on `stream`, the five required outputs are copied back and the stream is synchronised before
+ * the call returns -- this is the one entry point that synchronises.  Optional outputs and
+ * temperature_per_seq are not available here (SPEC_ERR_UNSUPPORTED when set).
+ */
+int32_t spec_host_staging_bytes(const SpecIn *in, int64_t *bytes);
+int32_t spec_verify_host(const SpecIn *in, const SpecOut *out, int32_t algorithm, void *dev_buf,
+                         int64_t dev_bytes, void *stream);
+
 /* Launch plan chosen for a vocabulary size and dtype (host-only query, for benchmarks and tests):
  * CTAs per cluster, tokens per CTA slice, dynamic shared memory bytes per CTA, threads per CTA. */
 int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, int32_t *slice_len,

@@ -25,7 +25,7 @@ SPEC_F32, SPEC_BF16 = 0, 1
 ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_DTYPE",
           -4: "SPEC_ERR_PARAM", -5: "SPEC_ERR_WORKSPACE", -6: "SPEC_ERR_UNSUPPORTED", -7: "SPEC_ERR_CUDA"}
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
-           "spec_sample_bonus", "spec_query_plan")
+           "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host")
 
 
 class SpecIn(C.Structure):
@@ -74,6 +74,11 @@ def load_library(path: str = LIB_PATH):
                                       C.c_void_p, C.c_int64, C.c_void_p]
     lib.spec_query_plan.restype = C.c_int32
     lib.spec_query_plan.argtypes = [C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 4
+    lib.spec_host_staging_bytes.restype = C.c_int32
+    lib.spec_host_staging_bytes.argtypes = [C.POINTER(SpecIn), C.POINTER(C.c_int64)]
+    lib.spec_verify_host.restype = C.c_int32
+    lib.spec_verify_host.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_int32, C.c_void_p, C.c_int64,
+                                     C.c_void_p]
     _lib = lib
     return lib
 
@@ -273,51 +278,62 @@ def sample_bonus(weights, u, want_margin=False, stream=None):
 
 
 class HostVerifier:
-    """End-to-end call for callers whose logits live in (pinned) host memory.
+    """End-to-end call for callers whose logits live in host memory (``spec_verify_host``).
 
-    Owns device staging buffers for one batch shape.  ``run`` copies the inputs host->device, enqueues
-    the verifier, copies the decisions device->host and synchronises the stream once.
+    Owns the device staging buffer for one batch shape and pinned host result arrays.  ``run`` hands
+    host pointers to the library, which copies the inputs host->device, runs the verifier, copies the
+    decisions device->host and synchronises the stream before returning.
     """
 
-    def __init__(self, B, N, V, logits_dtype=torch.bfloat16, device="cuda", algorithm="specinfer"):
+    ALGORITHMS = {"specinfer": 0, "traversal": 1}
+
+    def __init__(self, B, N, V, logits_dtype=torch.bfloat16, device="cuda", algorithm="specinfer",
+                 per_sequence_topology=False):
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
-        load_library()
+        self.lib = load_library()
         self.device = torch.device(device)
-        self.algorithm = algorithm
+        self.algorithm = self.ALGORITHMS[algorithm]
         self.shape = (B, N, V)
-        d = self.device
-        self.zp = torch.empty((B, N, V), dtype=logits_dtype, device=d)
-        self.zq = torch.empty((B, N, V), dtype=logits_dtype, device=d)
-        self.parent = torch.empty(N, dtype=torch.int32, device=d)
-        self.token = torch.empty((B, N), dtype=torch.int32, device=d)
-        self.ua = torch.empty((B, N), dtype=torch.float32, device=d)
-        self.ub = torch.empty((B, N), dtype=torch.float32, device=d)
-        self.out = alloc_outputs(B, N, V, d)
-        self.host_out = {k: torch.empty_like(getattr(self.out, k), device="cpu").pin_memory()
-                         for k in ("accepted_node", "accept_len", "out_tokens", "bonus_token", "status")}
-        self.ws = Workspace(d)
-        self.stream = torch.cuda.Stream(device=d)
+        self.dtype = logits_dtype
+        self.per_seq = per_sequence_topology
+        probe = SpecIn(B, N, V, SPEC_F32 if logits_dtype == torch.float32 else SPEC_BF16, None, None, N * V, V,
+                       None, N if per_sequence_topology else 0, None, 1.0, 0, 1.0, None, None, None)
+        n = C.c_int64()
+        _check(self.lib.spec_host_staging_bytes(C.byref(probe), C.byref(n)), "spec_host_staging_bytes")
+        self.staging = torch.empty(int(n.value) + 256, dtype=torch.uint8, device=self.device)
+        self.host_out = {k: torch.empty(shape, dtype=torch.int32).pin_memory()
+                         for k, shape in (("accepted_node", (B,)), ("accept_len", (B,)), ("out_tokens", (B, N)),
+                                          ("bonus_token", (B,)), ("status", (B,)))}
+        self.stream = torch.cuda.Stream(device=self.device)
 
     def h2d_bytes(self) -> int:
-        return sum(t.numel() * t.element_size() for t in (self.zp, self.zq, self.parent, self.token, self.ua, self.ub))
+        B, N, V = self.shape
+        esz = 4 if self.dtype == torch.float32 else 2
+        return 2 * B * N * V * esz + (B if self.per_seq else 1) * N * 4 + 3 * B * N * 4
 
     def d2h_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in self.host_out.values())
 
     def run(self, target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0, top_k=0,
             top_p=1.0):
-        with torch.cuda.stream(self.stream):
-            self.zp.copy_(target_logits, non_blocking=True)
-            self.zq.copy_(draft_logits, non_blocking=True)
-            self.parent.copy_(parent, non_blocking=True)
-            self.token.copy_(token, non_blocking=True)
-            self.ua.copy_(u_accept, non_blocking=True)
-            self.ub.copy_(u_bonus, non_blocking=True)
-            fn = verify_specinfer if self.algorithm == "specinfer" else verify_traversal
-            fn(self.zp, self.zq, self.parent, self.token, self.ua, self.ub, temperature, top_k, top_p,
-               outputs=self.out, workspace=self.ws, stream=self.stream)
-            for k, h in self.host_out.items():
-                h.copy_(getattr(self.out, k), non_blocking=True)
-        self.stream.synchronize()
-        return self.host_out
+        """All arguments are host tensors (pinned for asynchronous copies).  Returns pinned host results."""
+        B, N, V = self.shape
+        for name, t in (("target_logits", target_logits), ("draft_logits", draft_logits), ("parent", parent),
+                        ("token", token), ("u_accept", u_accept), ("u_bonus", u_bonus)):
+            if t.is_cuda or not t.is_contiguous():
+                raise RuntimeError(f"{name} must be a contiguous host tensor")
+        if tuple(target_logits.shape) != (B, N, V) or target_logits.dtype != self.dtype:
+            raise RuntimeError("logits do not match the shape / dtype this verifier was built for")
+        si = SpecIn(B, N, V, SPEC_F32 if self.dtype == torch.float32 else SPEC_BF16, _ptr(target_logits),
+                    _ptr(draft_logits), N * V, V, _ptr(parent), N if parent.dim() == 2 else 0, _ptr(token),
+                    float(temperature), int(top_k), float(top_p), None, _ptr(u_accept), _ptr(u_bonus))
+        h = self.host_out
+        so = SpecOut(_ptr(h["accepted_node"]), _ptr(h["accept_len"]), _ptr(h["out_tokens"]), _ptr(h["bonus_token"]),
+                     _ptr(h["status"]), None, None, None, None, None)
+        base = self.staging.data_ptr()
+        off = (-base) % 256
+        _check(self.lib.spec_verify_host(C.byref(si), C.byref(so), self.algorithm, C.c_void_p(base + off),
+                                         self.staging.numel() - off, C.c_void_p(self.stream.cuda_stream)),
+               "spec_verify_host")
+        return h

@@ -472,6 +472,7 @@ __global__ void __launch_bounds__(NT, 1) spec_node_kernel(const KParams P)
     const int tid = threadIdx.x;
     const int SL = P.SL;
     __shared__ Shared S;
+    cluster.barrier_arrive();            // peers must be running before their shared memory is written
 
     float *ep = (float *)dyn_smem;
     float *eq = ep + SL;
@@ -591,6 +592,7 @@ __global__ void __launch_bounds__(NT, 1) spec_node_kernel(const KParams P)
     }
 
     // ---- exchange 1: per-slice max / sums (+ w_in from rank 0) -----------------------------------
+    cluster.barrier_wait();
     cluster_allgather(cluster, S, parity, v, NX);
     double (*X)[NX] = S.xchg[parity];
     parity ^= 1;
@@ -967,6 +969,7 @@ __global__ void __launch_bounds__(NT, 1) spec_probs_kernel(const TParams P)
         v[1] = red[0]; v[2] = red[1];
     }
     v[0] = (double)m; v[6] = any_nan ? 1.0 : 0.0;
+    cluster.sync();                      // peers must be running before their shared memory is written
     cluster_allgather(cluster, S, 0, v, NX);
     double (*X)[NX] = S.xchg[0];
     double mg = -CUDART_INF;
@@ -1046,6 +1049,7 @@ __global__ void __launch_bounds__(NT, 1) spec_bonus_kernel(const BParams P)
     }
     double red[1] = {acc};
     block_sum<1>(S, red);
+    cluster.sync();                      // peers must be running before their shared memory is written
     cluster_allgather(cluster, S, 0, red, 1);
     double (*X)[NX] = S.xchg[0];
     double tot = 0.0;
@@ -1200,6 +1204,42 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     return SPEC_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// host-buffer entry point: staging layout inside the caller's device buffer
+// ------------------------------------------------------------------------------------------------
+struct HostLayout {
+    int64_t zp, zq, parent, token, ua, ub, acc, len, toks, bonus, status, ws, total;
+    int64_t logit_bytes, parent_bytes, bn4, b4;
+};
+
+inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
+
+HostLayout host_layout(const SpecIn *in)
+{
+    HostLayout L = {};
+    const int64_t esz = in->logits_dtype == SPEC_BF16 ? 2 : 4;
+    L.logit_bytes = (int64_t)in->B * in->N * in->V * esz;
+    L.parent_bytes = (in->topo_seq_stride ? (int64_t)in->B : 1) * in->N * 4;
+    L.bn4 = (int64_t)in->B * in->N * 4;
+    L.b4 = (int64_t)in->B * 4;
+    int64_t o = 0;
+    L.zp = o; o += up256(L.logit_bytes);
+    L.zq = o; o += up256(L.logit_bytes);
+    L.parent = o; o += up256(L.parent_bytes);
+    L.token = o; o += up256(L.bn4);
+    L.ua = o; o += up256(L.bn4);
+    L.ub = o; o += up256(L.bn4);
+    L.acc = o; o += up256(L.b4);
+    L.len = o; o += up256(L.b4);
+    L.toks = o; o += up256(L.bn4);
+    L.bonus = o; o += up256(L.b4);
+    L.status = o; o += up256(L.b4);
+    L.ws = o; o += up256(workspace_need(in));
+    L.total = o;
+    return L;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1267,6 +1307,60 @@ int32_t spec_sample_bonus(const float *weights, int32_t R, int32_t V, const floa
     if (!make_plan(V, 4, &pl)) return SPEC_ERR_UNSUPPORTED;
     BParams bp = {R, V, pl.SL, weights, u, token, margin};
     return launch_clustered(spec_bonus_kernel, R, pl, (cudaStream_t)stream, &bp);
+}
+
+
+int32_t spec_host_staging_bytes(const SpecIn *in, int64_t *bytes)
+{
+    if (!in || !bytes) return SPEC_ERR_NULL;
+    int rc = check_in(in, false);
+    if (rc) return rc;
+    *bytes = host_layout(in).total;
+    return SPEC_OK;
+}
+
+int32_t spec_verify_host(const SpecIn *in, const SpecOut *out, int32_t algorithm, void *dev_buf,
+                         int64_t dev_bytes, void *stream)
+{
+    int rc = check_in(in, true);
+    if (rc) return rc;
+    if (!out || !out->accepted_node || !out->accept_len || !out->out_tokens || !out->bonus_token || !out->status)
+        return SPEC_ERR_NULL;
+    if (out->residual || out->node_thr || out->node_w_in || out->node_features || out->margin)
+        return SPEC_ERR_UNSUPPORTED;
+    if (algorithm != 0 && algorithm != 1) return SPEC_ERR_PARAM;
+    if (in->temperature_per_seq) return SPEC_ERR_UNSUPPORTED;
+    if (in->node_stride != in->V || in->seq_stride != (int64_t)in->N * in->V) return SPEC_ERR_SHAPE;
+    if (in->topo_seq_stride != 0 && in->topo_seq_stride != in->N) return SPEC_ERR_SHAPE;
+    const HostLayout L = host_layout(in);
+    if (!dev_buf || ((uintptr_t)dev_buf & 255) || dev_bytes < L.total) return SPEC_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *d = (unsigned char *)dev_buf;
+    bool ok = true;
+    ok &= cudaMemcpyAsync(d + L.zp, in->target_logits, (size_t)L.logit_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + L.zq, in->draft_logits, (size_t)L.logit_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + L.parent, in->parent, (size_t)L.parent_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + L.token, in->token, (size_t)L.bn4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + L.ua, in->u_accept, (size_t)L.bn4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d + L.ub, in->u_bonus, (size_t)L.bn4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    SpecIn din = *in;
+    din.target_logits = d + L.zp; din.draft_logits = d + L.zq;
+    din.parent = (const int32_t *)(d + L.parent); din.token = (const int32_t *)(d + L.token);
+    din.u_accept = (const float *)(d + L.ua); din.u_bonus = (const float *)(d + L.ub);
+    SpecOut dout = {};
+    dout.accepted_node = (int32_t *)(d + L.acc); dout.accept_len = (int32_t *)(d + L.len);
+    dout.out_tokens = (int32_t *)(d + L.toks); dout.bonus_token = (int32_t *)(d + L.bonus);
+    dout.status = (int32_t *)(d + L.status);
+    rc = verify_common(&din, &dout, d + L.ws, L.total - L.ws, stream, algorithm == 0 ? MODE_SPECINFER : MODE_TRAVERSAL);
+    if (rc) return rc;
+    ok &= cudaMemcpyAsync(out->accepted_node, dout.accepted_node, (size_t)L.b4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out->accept_len, dout.accept_len, (size_t)L.b4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out->out_tokens, dout.out_tokens, (size_t)L.bn4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out->bonus_token, dout.bonus_token, (size_t)L.b4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(out->status, dout.status, (size_t)L.b4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    return SPEC_OK;
 }
 
 }  // extern "C"

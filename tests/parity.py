@@ -124,8 +124,8 @@ def check_batch(batch, algo, full=True) -> Tally:
     internal = np.zeros(N, bool); internal[parent[1:]] = True
     assert np.abs(feats[..., 0] - sp[..., 3]).max() < 1e-4
     assert np.abs(feats[..., 2] - sp[..., 4]).max() < PROB_TOL
-    assert np.abs(feats[:, internal, 1] - sq[:, internal, 3]).max() < 1e-4
-    assert np.abs(feats[:, internal, 3] - sq[:, internal, 4]).max() < PROB_TOL
+    assert np.abs(feats[:, internal, 1] - sq[:, internal, 3]).max(initial=0.0) < 1e-4
+    assert np.abs(feats[:, internal, 3] - sq[:, internal, 4]).max(initial=0.0) < PROB_TOL
     mg = got.margin.cpu().numpy()
     ua = inp.u_accept.astype(np.float64)
     ref_thr = ratio if algo == "specinfer" else w_fin
