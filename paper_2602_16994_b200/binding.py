@@ -242,6 +242,40 @@ def verify_traversal(target_logits, draft_logits, parent, token, u_accept, u_bon
                    node_thr=node_thr, node_w_in=node_w_in, features=features, margin=margin)
 
 
+class PreparedVerify:
+    """One verification call with its arguments marshalled once: ``launch()`` is a single C call.
+
+    For loops that verify the same buffers again and again (a decoding loop reusing its logits
+    buffers, a benchmark).  The tensors are kept alive by this object.  ``launch`` may be recorded
+    into a CUDA graph after one ordinary call on the device (the first call sets kernel attributes).
+    """
+
+    def __init__(self, algorithm, target_logits, draft_logits, parent, token, u_accept, u_bonus,
+                 temperature=1.0, top_k=0, top_p=1.0, temperature_per_seq=None, outputs=None, workspace=None,
+                 **alloc):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
+        self.fn = getattr(self.lib, {"specinfer": "spec_verify_specinfer",
+                                     "traversal": "spec_verify_traversal"}[algorithm])
+        self.name = algorithm
+        self.spec_in, self.keep = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus,
+                                           temperature, top_k, top_p, temperature_per_seq)
+        B, N, V = self.spec_in.B, self.spec_in.N, self.spec_in.V
+        dev = target_logits.device
+        self.outputs = outputs if outputs is not None else alloc_outputs(B, N, V, dev, **alloc)
+        self.spec_out = self.outputs.as_struct()
+        self.workspace = workspace or _ws_for(dev)
+        self.ws_ptr, self.ws_size = self.workspace.get(workspace_bytes(self.spec_in))
+        self._in_ref, self._out_ref = C.byref(self.spec_in), C.byref(self.spec_out)
+
+    def launch(self, stream=None):
+        rc = self.fn(self._in_ref, self._out_ref, self.ws_ptr, self.ws_size, _stream_ptr(stream))
+        if rc != 0:
+            _check(rc, "spec_verify_" + self.name)
+        return self.outputs
+
+
 def tree_probs(logits, which=0, temperature=1.0, top_k=0, top_p=1.0, temperature_per_seq=None,
                want_probs=True, want_stats=True, stream=None):
     """Sampling distribution of every row of ``logits`` [B,N,V].  Returns (probs or None, stats or None)."""

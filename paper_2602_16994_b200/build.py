@@ -8,6 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 SRC = [os.path.join(HERE, "csrc", "specverify.cu")]
+DEPS = [os.path.join(HERE, "csrc", f) for f in ("common.cuh", "verify.cuh", "rowops.cuh")]
 LIB = os.path.join(HERE, "libspecverify.so")
 HEADERS = [os.path.join(ROOT, "include", "specverify.h")]
 
@@ -16,7 +17,7 @@ def stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(f) > t for f in SRC + HEADERS)
+    return any(os.path.getmtime(f) > t for f in SRC + DEPS + HEADERS)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

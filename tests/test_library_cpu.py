@@ -101,10 +101,11 @@ def test_other_entry_points_reject_bad_arguments(lib):
 
 def test_query_plan():
     p = binding.query_plan(128256)
-    assert p["cluster_size"] == 8 and p["slice_len"] % 64 == 0 and p["slice_len"] * 8 >= 128256
-    assert p["smem_bytes"] <= 227 * 1024
+    assert p["cluster_size"] == 8 and p["slice_len"] % 8 == 0 and p["slice_len"] * 8 >= 128256
+    assert p["smem_bytes"] <= 113 * 1024 and p["threads"] == 256     # two CTAs per SM
     assert binding.query_plan(1000, 0)["cluster_size"] == 1
-    assert binding.query_plan(262144)["cluster_size"] == 16
+    big = binding.query_plan(262144)
+    assert big["slice_len"] * big["cluster_size"] >= 262144 and big["smem_bytes"] <= 227 * 1024
 
 
 def test_binding_refuses_to_run_without_a_gpu():
