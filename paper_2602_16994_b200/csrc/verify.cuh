@@ -135,7 +135,8 @@ __device__ __forceinline__ void mask_chunk(float (&z)[8], int nvalid, bool has_c
     }
 }
 
-// e[k] = 2^(z[k] s - of) for the 8 logits of a chunk, of the thread's reference for this row (an
+// e[k] = 2^(z[k] s - of) for the 8 logits of a chunk (the large product z s_hi - of is formed first, in
+// one rounding, so that the exponent's error is relative to the exponent and not to of), of the thread's reference for this row (an
 // integer-valued float); returns sum e.  FEAT: also sx += sum e x with x the exponent.
 template <bool FEAT>
 __device__ __forceinline__ float exp_chunk(const float (&z)[8], float s_hi, float s_lo, float of, float (&e)[8],
@@ -144,7 +145,7 @@ __device__ __forceinline__ float exp_chunk(const float (&z)[8], float s_hi, floa
     float sum = 0.f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        float x = fmaf(z[k], s_hi, fmaf(z[k], s_lo, -of));
+        float x = fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of));
         if (FEAT) x = fmaxf(x, -200.f);
         e[k] = ex2_approx(x);
         sum += e[k];
@@ -213,7 +214,7 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
             (O) = fminf(fmaxf(ceilf(zm_ * s_hi), -1.0e9f), 1.0e9f);                                          \
             (SET) = true;                                                                                    \
         }                                                                                                    \
-        const float xm_ = fmaf(zm_, s_hi, fmaf(zm_, s_lo, -(O)));                                            \
+        const float xm_ = fmaf(zm_, s_lo, fmaf(zm_, s_hi, -(O)));                                            \
         if (xm_ > 60.f && xm_ < CUDART_INF_F) {                                                              \
             const float kf_ = fminf(ceilf(xm_), 1.0e9f);                                                     \
             const float f_ = pow2i(-(int)fminf(kf_, 200.f));                                                 \
@@ -229,7 +230,7 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
         }                                                                                                    \
         float e8_[8];                                                                                        \
         (SUM) += exp_chunk<FEAT>(Z, s_hi, s_lo, (O), e8_, (SX));                                             \
-        if (FEAT) (BX) = fmaxf((BX), fmaf(zm_, s_hi, fmaf(zm_, s_lo, -(O))));                                \
+        if (FEAT) (BX) = fmaxf((BX), fmaf(zm_, s_lo, fmaf(zm_, s_hi, -(O))));                                \
         if (ISREG) {                                                                                         \
             _Pragma("unroll") for (int k_ = 0; k_ < 8; ++k_) E[(J)][k_] = e8_[k_];                           \
         } else {                                                                                             \
@@ -853,13 +854,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
                     const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
                     load_e8(d, NCONS, p);
                     load_e8(d + 2 * NCONS, NCONS, q);
-                    const float r = warp_sum(residual_chunk(p, q, gh_c, gl_c) * phi_t);
-                    if (lane == 0) S.wtile[warp][i] = (double)r;
+                    const double r = warp_sum((double)(residual_chunk(p, q, gh_c, gl_c) * phi_t));
+                    if (lane == 0) S.wtile[warp][i] = r;
                 }
 #pragma unroll
                 for (int jr = 0; jr < RT; ++jr) {
-                    const float r = warp_sum(residual_chunk(ep[jr], eq[jr], gh_c, gl_c) * phi_t);
-                    if (lane == 0) S.wtile[warp][nsm + jr] = (double)r;
+                    const double r = warp_sum((double)(residual_chunk(ep[jr], eq[jr], gh_c, gl_c) * phi_t));
+                    if (lane == 0) S.wtile[warp][nsm + jr] = r;
                 }
                 bar_sync(1, NCONS);
                 // tile, then warp inside the tile, then lane inside the warp, then token inside the chunk
