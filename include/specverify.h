@@ -132,6 +132,31 @@ int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, in
                               void *stream);
 
 /*
+ * SpecInfer verification for callers that cannot allocate device memory.  The paper has no
+ * counterpart to this entry point: it exists for hosts of this library that are handed their
+ * device buffers by someone else and may not call cudaMalloc themselves -- a plugin running inside
+ * an inference server whose memory pool is closed to it, a process under a fixed memory budget, or
+ * code that runs where an allocation would stall or fail (a latency-critical decoding loop, a
+ * region in which the allocator is locked).  Same inputs, outputs and results as
+ * spec_verify_specinfer, but no `ws` argument: the scratch memory is an array of
+ * SPEC_STATIC_WS_BYTES bytes inside the library image, present on every GPU that has loaded the
+ * library until the process exits.
+ *   - Limit: B * N <= SPEC_STATIC_MAX_NODES (tree nodes summed over the batch); larger shapes
+ *     return SPEC_ERR_WORKSPACE and nothing is enqueued.  V is not limited by the scratch.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current) before it enqueues anything; make that first call outside any stream
+ *     capture.  No call allocates or frees memory.
+ *   - Every call uses the same array, which still holds the previous call's records when the next
+ *     one starts; the call clears the parts that must start empty (the published weights and the
+ *     arrival counters) on `stream` itself.  Two calls that can overlap on the GPU (different
+ *     streams without an ordering between them) race on the array: serialise them, or give the
+ *     others a workspace through spec_verify_specinfer.
+ */
+#define SPEC_STATIC_MAX_NODES 4096
+#define SPEC_STATIC_WS_BYTES (640 * 1024)
+int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void *stream);
+
+/*
  * Traversal Verification (Section 3.2, bottom-up; block verification of Section 3.1 on one
  * path).  Weights flow down: a child with token x gets min(1, w P(x)/q(x)) from its parent's
  * current (w, P); a node is tested (u_accept < w) only after all its child subtrees were

@@ -25,7 +25,8 @@ SPEC_F32, SPEC_BF16 = 0, 1
 ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR_DTYPE",
           -4: "SPEC_ERR_PARAM", -5: "SPEC_ERR_WORKSPACE", -6: "SPEC_ERR_UNSUPPORTED", -7: "SPEC_ERR_CUDA"}
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
-           "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host")
+           "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
+           "spec_verify_specinfer_static")
 
 
 class SpecIn(C.Structure):
@@ -69,6 +70,8 @@ def load_library(path: str = LIB_PATH):
         f = getattr(lib, name)
         f.restype = C.c_int32
         f.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_void_p, C.c_int64, C.c_void_p]
+    lib.spec_verify_specinfer_static.restype = C.c_int32
+    lib.spec_verify_specinfer_static.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_void_p]
     lib.spec_sample_bonus.restype = C.c_int32
     lib.spec_sample_bonus.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_int64, C.c_void_p]
@@ -229,6 +232,25 @@ def verify_specinfer(target_logits, draft_logits, parent, token, u_accept, u_bon
                  temperature_per_seq)
     return _verify("spec_verify_specinfer", m, outputs, workspace, stream, residual=residual,
                    node_thr=node_thr, features=features, margin=margin)
+
+
+def verify_specinfer_static(target_logits, draft_logits, parent, token, u_accept, u_bonus, outputs,
+                            temperature=1.0, top_k=0, top_p=1.0, stream=None):
+    """SpecInfer verification through ``spec_verify_specinfer_static``: the library's built-in scratch
+    array is used, so neither this wrapper nor the library allocates anything.  The caller owns every
+    buffer, ``outputs`` (a ``VerifyOutputs``) included.  Only for B * N up to 4096 nodes; calls that may
+    overlap on the GPU must not share this entry point.  Make the first call on a device outside any
+    stream capture.
+    """
+    lib = load_library()
+    if not torch.cuda.is_available():
+        raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
+    si, keep = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+                        None)
+    so = outputs.as_struct()
+    _check(lib.spec_verify_specinfer_static(C.byref(si), C.byref(so), _stream_ptr(stream)),
+           "spec_verify_specinfer_static")
+    return outputs
 
 
 def verify_traversal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0,

@@ -357,6 +357,30 @@ HostLayout host_layout(const SpecIn *in)
     return L;
 }
 
+// ------------------------------------------------------------------------------------------------
+// scratch that lives inside the library image, for spec_verify_specinfer_static
+// ------------------------------------------------------------------------------------------------
+constexpr int64_t STATIC_WS_BYTES = 640 * 1024;
+static __device__ __align__(256) unsigned char g_static_ws[STATIC_WS_BYTES];
+
+// Device address of g_static_ws on the current device.  In host code the array's name is only a
+// handle for the runtime, never a device pointer, so the address is asked for once per device (with
+// that device current) and remembered.
+int static_ws_address(void **ptr)
+{
+    static void *addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(g_cache_mutex);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_ws) != cudaSuccess || !p) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+        addr[dev] = p;
+    }
+    *ptr = addr[dev];
+    return SPEC_OK;
+}
+
 }  // namespace
 }  // namespace specv
 
@@ -395,6 +419,17 @@ int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, in
 int32_t spec_verify_traversal(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream)
 {
     return verify_common(in, out, ws, ws_bytes, stream, MODE_TRAVERSAL);
+}
+
+int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void *stream)
+{
+    int rc = check_in(in, true);
+    if (rc) return rc;
+    if ((int64_t)in->B * in->N > SPEC_STATIC_MAX_NODES || ws_layout(in).total > STATIC_WS_BYTES) return SPEC_ERR_WORKSPACE;
+    void *ws = nullptr;
+    rc = static_ws_address(&ws);
+    if (rc) return rc;
+    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER);
 }
 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,
