@@ -114,7 +114,9 @@ int32_t spec_workspace_bytes(const SpecIn *in, int64_t *bytes);
  *   row_stats  optional [B,N,6] float: max of z/T, sum of kept exp(z/T - max), kept count,
  *              entropy (nats), largest probability, smallest kept logit value.
  * Only B, N, V, dtype, the logits of the chosen side, strides and the sampling parameters of `in`
- * are read.  Rows that are not finite produce NaN statistics and zero probabilities.
+ * are read (every row of the chosen side is read, whatever the tree).  With truncating parameters
+ * (top_k or top_p active) `ws` must be a workspace of spec_workspace_bytes(); otherwise it may be
+ * NULL.  Rows that are not finite produce NaN statistics and zero probabilities.
  */
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats,
                         void *ws, int64_t ws_bytes, void *stream);

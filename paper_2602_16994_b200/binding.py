@@ -311,8 +311,9 @@ def tree_probs(logits, which=0, temperature=1.0, top_k=0, top_p=1.0, temperature
                 float(temperature), int(top_k), float(top_p), _ptr(temperature_per_seq), None, None)
     probs = torch.empty((B, N, V), dtype=torch.float32, device=logits.device) if want_probs else None
     stats = torch.empty((B, N, 6), dtype=torch.float32, device=logits.device) if want_stats else None
-    _check(lib.spec_tree_probs(C.byref(si), int(which), _ptr(probs), _ptr(stats), None, 0, _stream_ptr(stream)),
-           "spec_tree_probs")
+    ws_ptr, ws_size = _ws_for(logits.device).get(workspace_bytes(si))       # holds the row cuts when truncating
+    _check(lib.spec_tree_probs(C.byref(si), int(which), _ptr(probs), _ptr(stats), ws_ptr, ws_size,
+                               _stream_ptr(stream)), "spec_tree_probs")
     return probs, stats
 
 

@@ -179,9 +179,10 @@ __device__ __forceinline__ float raw_max(const float *region, int SL, int dtype,
 // barrier, then writes 8 floats; step s writes bytes [16384 s, 16384 (s+1)) of the region while the
 // unread raw data starts at 2 SL + 8192 (s+1) >= 16384 (s+1) as long as a later step exists.
 __device__ __forceinline__ void widen_exp(float *region, int SL, int dtype, int n, float m, float cut,
-                                          float s_hi, float s_lo, double &sum_e, double &sum_ex)
+                                          float s_hi, float s_lo, double &sum_e, double &sum_ex, int &kept)
 {
     double acc_e = 0.0, acc_x = 0.0;
+    int nk = 0;
     if (dtype == SPEC_BF16) {
         const unsigned char *raw = raw_ptr(region, SL, dtype);
         int steps = (SL + NT * 8 - 1) / (NT * 8);
@@ -199,6 +200,7 @@ __device__ __forceinline__ void widen_exp(float *region, int SL, int dtype, int 
                 for (int k = 0; k < 8; ++k) {
                     float z = (k & 1) ? bf16_hi(w[k >> 1]) : bf16_lo(w[k >> 1]);
                     bool keep = (t0 + k < n) && (z >= cut);
+                    nk += keep ? 1 : 0;
                     float x;
                     float v = exp_scaled(keep ? z : -CUDART_INF_F, m, s_hi, s_lo, x);
                     e[k] = v;
@@ -224,6 +226,7 @@ __device__ __forceinline__ void widen_exp(float *region, int SL, int dtype, int 
             for (int k = 0; k < 4; ++k) {
                 float x;
                 bool keep = ((i * 4 + k) < n) && (zz[k] >= cut);
+                nk += keep ? 1 : 0;
                 float val = exp_scaled(keep ? zz[k] : -CUDART_INF_F, m, s_hi, s_lo, x);
                 e[k] = val;
                 pe += val;
@@ -236,6 +239,7 @@ __device__ __forceinline__ void widen_exp(float *region, int SL, int dtype, int 
     }
     sum_e = acc_e;
     sum_ex = acc_x;
+    kept = nk;
 }
 
 // Inverse CDF inside one slice.  Weights w_t = (ep[t] - gamma eq[t])+ (eq may be NULL: w = ep).
@@ -337,6 +341,8 @@ struct TParams {
     float T;
     const float *T_seq;
     float *probs, *stats;
+    const float *cut;        // optional [rows*2] smallest kept logit (target, draft) of every row
+    int which;
 };
 
 __global__ void __launch_bounds__(NT, 1) spec_probs_kernel(const TParams P)
@@ -377,11 +383,13 @@ __global__ void __launch_bounds__(NT, 1) spec_probs_kernel(const TParams P)
     double v[NX];
 #pragma unroll
     for (int i = 0; i < NX; ++i) v[i] = 0.0;
-    widen_exp(ep, SL, P.dtype, n, ref, -CUDART_INF_F, s_hi, s_lo, v[1], v[2]);
+    const float cutv = P.cut ? __ldg(P.cut + (long long)row_id * 2 + P.which) : -CUDART_INF_F;
+    int kept = 0;
+    widen_exp(ep, SL, P.dtype, n, ref, cutv, s_hi, s_lo, v[1], v[2], kept);
     {
-        double red[2] = {v[1], v[2]};
-        block_sum<2>(S, red);
-        v[1] = red[0]; v[2] = red[1];
+        double red[3] = {v[1], v[2], (double)kept};
+        block_sum<3>(S, red);
+        v[1] = red[0]; v[2] = red[1]; v[3] = red[2];
     }
     v[0] = (double)m; v[6] = any_nan ? 1.0 : 0.0;
     cluster.sync();                      // peers must be running before their shared memory is written
@@ -413,8 +421,10 @@ __global__ void __launch_bounds__(NT, 1) spec_probs_kernel(const TParams P)
                 double sp = S.scale_p[r];
                 if (sp > 0.0) h -= (sp / Z) * (0.6931471805599453 * X[r][2] + (log(sp) - log(Z)) * X[r][1]);
             }
-            st[0] = (float)(mg / T); st[1] = (float)Z; st[2] = (float)P.V;
-            st[3] = (float)h; st[4] = (float)(1.0 / Z); st[5] = -CUDART_INF_F;
+            double nkept = 0.0;
+            for (int r = 0; r < C; ++r) nkept += X[r][3];
+            st[0] = (float)(mg / T); st[1] = (float)Z; st[2] = (float)nkept;
+            st[3] = (float)h; st[4] = (float)(1.0 / Z); st[5] = cutv;
         }
     }
 }

@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "cut.cuh"
 #include "rowops.cuh"
 #include "specverify.h"
 #include "verify.cuh"
@@ -264,6 +265,21 @@ int launch_verify(const VPlan &pl, VParams &vp, cudaStream_t st)
     return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &vp);
 }
 
+// row cuts for truncating sampling parameters, written to `cut` ([B*N*2] floats)
+int launch_cuts(const SpecIn *in, float *cut, cudaStream_t st)
+{
+    cut::CParams cp = {};
+    cp.B = in->B; cp.N = in->N; cp.V = in->V; cp.dtype = in->logits_dtype; cp.top_k = in->top_k; cp.top_p = in->top_p;
+    cp.zp = in->target_logits; cp.zq = in->draft_logits;
+    cp.seq_stride = in->seq_stride; cp.node_stride = in->node_stride; cp.topo_stride = in->topo_seq_stride;
+    cp.parent = in->parent; cp.T = in->temperature; cp.T_seq = in->temperature_per_seq; cp.cut = cut;
+    const unsigned grid = (unsigned)(2ll * in->B * in->N);
+    if (in->logits_dtype == SPEC_BF16) cut::spec_row_cut_kernel<SPEC_BF16><<<grid, cut::NT, 0, st>>>(cp);
+    else cut::spec_row_cut_kernel<SPEC_F32><<<grid, cut::NT, 0, st>>>(cp);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    return SPEC_OK;
+}
+
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode)
 {
     int rc = check_in(in, true);
@@ -271,7 +287,6 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     if (!out || !out->accepted_node || !out->accept_len || !out->out_tokens || !out->bonus_token || !out->status)
         return SPEC_ERR_NULL;
     const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
-    if (trunc) return SPEC_ERR_UNSUPPORTED;
     const WsLayout L = ws_layout(in);
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
     VPlan pl;
@@ -283,6 +298,10 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         cudaGetLastError();
         return SPEC_ERR_CUDA;
     }
+    if (trunc) {
+        rc = launch_cuts(in, (float *)(w + L.cut), st);
+        if (rc) return rc;
+    }
     VParams vp = {};
     vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
     vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
@@ -292,7 +311,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
     vp.parent = in->parent; vp.token = in->token;
     vp.T = in->temperature; vp.T_seq = in->temperature_per_seq;
-    vp.cut = nullptr;
+    vp.cut = trunc ? (const float *)(w + L.cut) : nullptr;
     vp.u_accept = in->u_accept; vp.u_bonus = in->u_bonus;
     vp.rec = (NodeRec *)(w + L.rec);
     vp.w_pub = (unsigned long long *)(w + L.pub);
@@ -435,20 +454,37 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,
                         int64_t ws_bytes, void *stream)
 {
-    (void)ws; (void)ws_bytes;
     int rc = check_in(in, false);
     if (rc) return rc;
     if (which != 0 && which != 1) return SPEC_ERR_PARAM;
     const void *z = which ? in->draft_logits : in->target_logits;
     if (!z || (!probs && !row_stats)) return SPEC_ERR_NULL;
-    if (in->top_k > 0 && in->top_k < in->V) return SPEC_ERR_UNSUPPORTED;
-    if (in->top_p < 1.f) return SPEC_ERR_UNSUPPORTED;
+    const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
+    const float *cutp = nullptr;
+    if (trunc) {
+        // the cuts of every row of the chosen side go to the workspace; the tree is not consulted here,
+        // so the kernel is told that every node has children (parent = NULL is not read for which = 0)
+        const WsLayout L = ws_layout(in);
+        if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
+        cut::CParams cp = {};
+        cp.B = in->B; cp.N = in->N; cp.V = in->V; cp.dtype = in->logits_dtype; cp.top_k = in->top_k; cp.top_p = in->top_p;
+        cp.zp = z; cp.zq = z; cp.seq_stride = in->seq_stride; cp.node_stride = in->node_stride;
+        cp.topo_stride = 0; cp.parent = nullptr; cp.T = in->temperature; cp.T_seq = in->temperature_per_seq;
+        cp.cut = (float *)((unsigned char *)ws + L.cut);
+        cp.only_target = 1;
+        const unsigned grid = (unsigned)(2ll * in->B * in->N);
+        if (in->logits_dtype == SPEC_BF16) cut::spec_row_cut_kernel<SPEC_BF16><<<grid, cut::NT, 0, (cudaStream_t)stream>>>(cp);
+        else cut::spec_row_cut_kernel<SPEC_F32><<<grid, cut::NT, 0, (cudaStream_t)stream>>>(cp);
+        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+        cutp = cp.cut;
+    }
     RowPlan pl;
     if (!make_row_plan(in->V, 4, &pl)) return SPEC_ERR_UNSUPPORTED;
     rowops::TParams tp = {};
     tp.rows = in->B * in->N; tp.N = in->N; tp.V = in->V; tp.dtype = in->logits_dtype; tp.SL = pl.SL;
     tp.z = z; tp.seq_stride = in->seq_stride; tp.node_stride = in->node_stride;
     tp.T = in->temperature; tp.T_seq = in->temperature_per_seq; tp.probs = probs; tp.stats = row_stats;
+    tp.cut = cutp; tp.which = 0;
     rc = prepare_kernel(rowops::spec_probs_kernel, pl.C, pl.smem);
     if (rc) return rc;
     return launch_clustered(rowops::spec_probs_kernel, tp.rows * pl.C, pl.C, rowops::NT, pl.smem, (cudaStream_t)stream, &tp);

@@ -205,3 +205,95 @@ def test_host_buffer_api_matches_device_api():
     np.testing.assert_array_equal(out["accepted_node"].numpy(), ref.accepted_node)
     np.testing.assert_array_equal(out["out_tokens"].numpy(), ref.out_tokens)
     assert hv.h2d_bytes() > 2 * w.B * w.N * w.V * 2 and hv.d2h_bytes() > 0
+
+
+# ---------------------------------------------------------------------------------------------
+# truncated sampling distributions (top-k / top-p)
+# ---------------------------------------------------------------------------------------------
+TRUNC = [dict(top_k=50), dict(top_p=0.95), dict(top_k=200, top_p=0.9), dict(top_k=1), dict(top_p=0.5)]
+
+
+@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (4099, torch.bfloat16), (128256, torch.bfloat16)])
+@pytest.mark.parametrize("trunc", TRUNC, ids=lambda d: "_".join(f"{k}{v}" for k, v in d.items()))
+def test_tree_probs_truncated(V, dtype, trunc):
+    g = torch.Generator(device="cuda").manual_seed(11)
+    z = (torch.randn((2, 3, V), generator=g, device="cuda") * 3).to(dtype)
+    z[0, 0, : V // 2] = z[0, 0, V // 2: 2 * (V // 2)]          # exact ties everywhere in one row
+    z[1, 1, 5] = -0.0
+    z[1, 1, 6] = 0.0
+    for T in (1.0, 0.6):
+        probs, stats = binding.tree_probs(z, 0, temperature=T, **trunc)
+        torch.cuda.synchronize()
+        zb = z.cpu()
+        bits = zb.view(torch.int16).numpy().view(np.uint16) if dtype == torch.bfloat16 else zb.numpy()
+        inp = oracle.TreeInputs(bits, bits, np.array([-1, 0, 0], np.int32), np.zeros((2, 3), np.int32),
+                                np.zeros((2, 3), np.float32), np.zeros((2, 3), np.float32), temperature=T,
+                                top_k=trunc.get("top_k", 0), top_p=trunc.get("top_p", 1.0))
+        rp, rs, _ = oracle.tree_probs(inp, 0)
+        sure = rs[..., 5] >= 1e-6                      # rows whose nucleus boundary is not within 1e-6 of top_p
+        assert sure.mean() > 0.8
+        got = probs.cpu().numpy()
+        st = stats.cpu().numpy().astype(np.float64)
+        assert np.abs(got - rp)[sure].max() < PROB_TOL
+        np.testing.assert_array_equal(st[..., 2][sure], rs[..., 2][sure])          # kept count
+        np.testing.assert_array_equal(st[..., 5][sure], rs[..., 6][sure].astype(np.float32))   # threshold logit
+
+
+TRUNC_SHAPES = [
+    Workload("t_v1000_f32_k", 6, 1000, "f32", 2, 0, 3, 1.0, temperature=0.8, top_k=20),
+    Workload("t_v4100_bf16_p", 5, 4100, "bf16", 3, 1, 2, 0.7, temperature=0.6, top_p=0.95),
+    Workload("t_v32000_bf16_kp", 4, 32000, "bf16", 4, 1, 3, 1.0, temperature=0.7, top_k=100, top_p=0.9),
+    Workload("t_v151936_bf16_p", 2, 151936, "bf16", 8, 0, 2, 0.7, temperature=0.6, top_p=0.95),
+    Workload("t_v128256_bf16_k", 2, 128256, "bf16", 8, 2, 2, 1.2, temperature=0.3, top_k=50),
+]
+
+
+def _unsure_sequences(inp):
+    """Sequences with a row whose nucleus boundary lies within 1e-6 of top_p (either side may keep or
+    drop the boundary group there)."""
+    _, sp, _ = oracle.tree_probs(inp, 0, want_probs=False)
+    _, sq, _ = oracle.tree_probs(inp, 1, want_probs=False)
+    parent = inp.parent if inp.parent.ndim == 1 else inp.parent[0]
+    internal = np.zeros(parent.shape[0], bool); internal[parent[1:]] = True
+    return (sp[..., 5] < 1e-6).any(1) | (sq[:, internal, 5] < 1e-6).any(1)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("w", TRUNC_SHAPES, ids=lambda w: w.name)
+def test_truncated_verification(algo, w):
+    batch = make_batch(w, seed=2, device="cuda")
+    inp = oracle_inputs(batch)
+    unsure = _unsure_sequences(inp)
+    assert unsure.mean() < 0.5
+    keep = [i for i in range(w.B) if not unsure[i]]
+    check_batch(batch.select(keep), algo)
+
+
+def test_cfg3_and_cfg5_sampled():
+    """The truncating workloads at full size in the bench's launch configuration; sampled sequences
+    against the oracle (SpecInfer + bonus, cfg5 with the selector features)."""
+    for name, picks in (("cfg3_qwen_b32", [0, 13, 31]), ("cfg5_serving_b128", [5, 77])):
+        w = WORKLOADS[name]
+        full = make_batch(w, seed=0, device="cuda")
+        got = binding.verify_specinfer(full.target_logits, full.draft_logits, full.parent, full.token, full.u_accept,
+                                       full.u_bonus, w.temperature, w.top_k, w.top_p, features=w.features)
+        torch.cuda.synchronize()
+        assert (got.status.cpu().numpy() == 0).all()
+        sub = full.select(picks)
+        inp, ref = run_oracle(sub, "specinfer")
+        unsure = _unsure_sequences(inp)
+        for i, b in enumerate(picks):
+            if unsure[i]:
+                continue
+            if got.accepted_node[b].item() != ref.accepted_node[i]:
+                assert min(ref.trace_margins[i], default=1.0) < 1e-6
+            elif got.bonus_token[b].item() != ref.bonus_token[i]:
+                assert ref.bonus_margin[i] < 1e-6
+            else:
+                np.testing.assert_array_equal(got.out_tokens[b].cpu().numpy(), ref.out_tokens[i])
+        if w.features:
+            _, sp, _ = oracle.tree_probs(inp, 0, want_probs=False)
+            f = got.node_features.cpu().numpy()[picks].astype(np.float64)
+            assert np.abs(f[..., 0] - sp[..., 3]).max() < 1e-4 and np.abs(f[..., 2] - sp[..., 4]).max() < PROB_TOL
+        del full, sub
+        torch.cuda.empty_cache()
