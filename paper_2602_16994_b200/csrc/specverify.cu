@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "cut.cuh"
 #include "rowops.cuh"
+#include "rowstat.cuh"
 #include "specverify.h"
 #include "verify.cuh"
 
@@ -149,7 +150,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 
 // workspace layout: node records | published weights + arrival counters (cleared per call) | row cuts
 struct WsLayout {
-    int64_t rec, pub, done, cut, clear_bytes, total;
+    int64_t rec, pub, done, cut, stat, clear_bytes, total;
 };
 WsLayout ws_layout(const SpecIn *in)
 {
@@ -162,6 +163,7 @@ WsLayout ws_layout(const SpecIn *in)
     L.clear_bytes = o - L.pub;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
+    L.stat = o; o += up256(nodes * 2 * (int64_t)sizeof(rowstat::RowStat));
     L.total = o;
     return L;
 }
@@ -265,19 +267,39 @@ int launch_verify(const VPlan &pl, VParams &vp, cudaStream_t st)
     return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &vp);
 }
 
-// row cuts for truncating sampling parameters, written to `cut` ([B*N*2] floats)
-int launch_cuts(const SpecIn *in, float *cut, cudaStream_t st)
+// row statistics (cut, reference, normaliser) of every row the verifiers read, or of every row of `z`
+// when no tree is given
+int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *parent, unsigned char *ws,
+                   const WsLayout &L, cudaStream_t st)
 {
-    cut::CParams cp = {};
-    cp.B = in->B; cp.N = in->N; cp.V = in->V; cp.dtype = in->logits_dtype; cp.top_k = in->top_k; cp.top_p = in->top_p;
-    cp.zp = in->target_logits; cp.zq = in->draft_logits;
-    cp.seq_stride = in->seq_stride; cp.node_stride = in->node_stride; cp.topo_stride = in->topo_seq_stride;
-    cp.parent = in->parent; cp.T = in->temperature; cp.T_seq = in->temperature_per_seq; cp.cut = cut;
-    const unsigned grid = (unsigned)(2ll * in->B * in->N);
-    if (in->logits_dtype == SPEC_BF16) cut::spec_row_cut_kernel<SPEC_BF16><<<grid, cut::NT, 0, st>>>(cp);
-    else cut::spec_row_cut_kernel<SPEC_F32><<<grid, cut::NT, 0, st>>>(cp);
-    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
-    return SPEC_OK;
+    const int esz = in->logits_dtype == SPEC_BF16 ? 2 : 4;
+    const int budget = 113 * 1024 - (int)sizeof(rowstat::Shared) - 2048;
+    int C = 1;
+    while (C <= rowstat::CMAXR && (long long)up((in->V + C - 1) / C, 8) * esz > budget) C <<= 1;
+    if (C > rowstat::CMAXR) return SPEC_ERR_UNSUPPORTED;
+    rowstat::RParams rp = {};
+    rp.B = in->B; rp.N = in->N; rp.V = in->V; rp.C = C; rp.dtype = in->logits_dtype;
+    rp.top_k = in->top_k; rp.top_p = in->top_p; rp.slice_len = up((in->V + C - 1) / C, 8);
+    rp.zp = zp; rp.zq = zq; rp.seq_stride = in->seq_stride; rp.node_stride = in->node_stride;
+    rp.topo_stride = in->topo_seq_stride; rp.parent = parent; rp.T = in->temperature; rp.T_seq = in->temperature_per_seq;
+    rp.stat = (rowstat::RowStat *)(ws + L.stat); rp.cut = (float *)(ws + L.cut);
+    const int smem = up(rp.slice_len * esz, 128);
+    const long long items = 2ll * in->B * in->N;
+    int rc, nc;
+    if (in->logits_dtype == SPEC_BF16) {
+        auto k = rowstat::spec_row_stat_kernel<SPEC_BF16>;
+        if ((rc = prepare_kernel(k, C, smem))) return rc;
+        nc = resident_clusters(k, C, rowstat::NT, smem);
+        if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
+        if (nc > items) nc = (int)items;
+        return launch_clustered(k, nc * C, C, rowstat::NT, smem, st, &rp);
+    }
+    auto k = rowstat::spec_row_stat_kernel<SPEC_F32>;
+    if ((rc = prepare_kernel(k, C, smem))) return rc;
+    nc = resident_clusters(k, C, rowstat::NT, smem);
+    if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
+    if (nc > items) nc = (int)items;
+    return launch_clustered(k, nc * C, C, rowstat::NT, smem, st, &rp);
 }
 
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode)
@@ -299,7 +321,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         return SPEC_ERR_CUDA;
     }
     if (trunc) {
-        rc = launch_cuts(in, (float *)(w + L.cut), st);
+        rc = launch_rowstat(in, in->target_logits, in->draft_logits, in->parent, w, L, st);
         if (rc) return rc;
     }
     VParams vp = {};
@@ -462,21 +484,12 @@ int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *ro
     const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
     const float *cutp = nullptr;
     if (trunc) {
-        // the cuts of every row of the chosen side go to the workspace; the tree is not consulted here,
-        // so the kernel is told that every node has children (parent = NULL is not read for which = 0)
+        // the cuts of every row of the chosen side go to slot 0 of every pair in the workspace
         const WsLayout L = ws_layout(in);
         if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
-        cut::CParams cp = {};
-        cp.B = in->B; cp.N = in->N; cp.V = in->V; cp.dtype = in->logits_dtype; cp.top_k = in->top_k; cp.top_p = in->top_p;
-        cp.zp = z; cp.zq = z; cp.seq_stride = in->seq_stride; cp.node_stride = in->node_stride;
-        cp.topo_stride = 0; cp.parent = nullptr; cp.T = in->temperature; cp.T_seq = in->temperature_per_seq;
-        cp.cut = (float *)((unsigned char *)ws + L.cut);
-        cp.only_target = 1;
-        const unsigned grid = (unsigned)(2ll * in->B * in->N);
-        if (in->logits_dtype == SPEC_BF16) cut::spec_row_cut_kernel<SPEC_BF16><<<grid, cut::NT, 0, (cudaStream_t)stream>>>(cp);
-        else cut::spec_row_cut_kernel<SPEC_F32><<<grid, cut::NT, 0, (cudaStream_t)stream>>>(cp);
-        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
-        cutp = cp.cut;
+        rc = launch_rowstat(in, z, z, nullptr, (unsigned char *)ws, L, (cudaStream_t)stream);
+        if (rc) return rc;
+        cutp = (const float *)((unsigned char *)ws + L.cut);
     }
     RowPlan pl;
     if (!make_row_plan(in->V, 4, &pl)) return SPEC_ERR_UNSUPPORTED;

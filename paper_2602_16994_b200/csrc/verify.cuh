@@ -33,7 +33,7 @@
 
 namespace specv {
 
-constexpr int RT = 4;        // tiles per thread whose e live in registers
+constexpr int RT = 4;        // tiles per thread whose e live in registers (the kernel names them one by one)
 constexpr int SMT = 6;       // further tiles per thread whose e live in shared memory
 constexpr int TMAX = RT + SMT;
 constexpr int CMAX = 16;     // CTAs per cluster (above 8: non-portable size)
@@ -201,13 +201,17 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
     return acc;
 }
 
-// Pass 1 for one row of one tile.  The tile's e go to the register tile E[J] (ISREG, a literal) or to
+// Pass 1 for one row of one tile.  The tile's e go to the register array DST (ISREG, a literal) or to
 // shared-memory slot SLOT.  O / SET / SUM / SX / BX: the thread's running reference for this row (an
 // integer-valued float), whether it is set, sum of e, sum of e x and largest exponent.  A chunk whose
 // largest exponent would exceed 60 moves the reference up and rescales what the thread has stored so
-// far by an exact power of two (rare: it takes logits 60 T / log2(e) above the first chunk's maximum).
-// NSM_DONE / J_DONE: how many shared-memory / register tiles of this row the thread has stored.
-#define SPECV_P1_ROW(Z, E, J, SLOT, ISREG, ROWOFF, NSM_DONE, J_DONE, O, SET, SUM, SX, BX)                    \
+// far by an exact power of two (rare: it takes logits 60 T / log2(e) above the first chunk's maximum):
+// the NSM_DONE shared-memory tiles of this row, and the register tiles named in RESCALE_REGS (a
+// statement list using the factor f_).  Register tiles are separate named arrays and every index is a
+// literal, so that they stay in registers.
+#define SPECV_SCALE8(A, F)                                                                                   \
+    do { _Pragma("unroll") for (int k_ = 0; k_ < 8; ++k_) A[k_] *= (F); } while (0)
+#define SPECV_P1_ROW(Z, DST, SLOT, ISREG, ROWOFF, NSM_DONE, RESCALE_REGS, O, SET, SUM, SX, BX)               \
     do {                                                                                                     \
         const float zm_ = max8(Z);                                                                           \
         if (!(SET) && zm_ > -CUDART_INF_F) {                                                                 \
@@ -218,8 +222,7 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
         if (xm_ > 60.f && xm_ < CUDART_INF_F) {                                                              \
             const float kf_ = fminf(ceilf(xm_), 1.0e9f);                                                     \
             const float f_ = pow2i(-(int)fminf(kf_, 200.f));                                                 \
-            _Pragma("unroll") for (int j_ = 0; j_ < RT; ++j_)                                                \
-                if (j_ < (J_DONE)) { _Pragma("unroll") for (int k_ = 0; k_ < 8; ++k_) E[j_][k_] *= f_; }     \
+            RESCALE_REGS                                                                                     \
             for (int j_ = 0; j_ < (NSM_DONE); ++j_) {                                                        \
                 float4 *d_ = es + (size_t)(j_ * 4 + (ROWOFF)) * NCONS + tid;                                 \
                 scale_f4(d_, f_); scale_f4(d_ + NCONS, f_);                                                  \
@@ -228,16 +231,16 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
             (SUM) *= f_;                                                                                     \
             (O) += kf_;                                                                                      \
         }                                                                                                    \
-        float e8_[8];                                                                                        \
-        (SUM) += exp_chunk<FEAT>(Z, s_hi, s_lo, (O), e8_, (SX));                                             \
-        if (FEAT) (BX) = fmaxf((BX), fmaf(zm_, s_lo, fmaf(zm_, s_hi, -(O))));                                \
         if (ISREG) {                                                                                         \
-            _Pragma("unroll") for (int k_ = 0; k_ < 8; ++k_) E[(J)][k_] = e8_[k_];                           \
+            (SUM) += exp_chunk<FEAT>(Z, s_hi, s_lo, (O), DST, (SX));                                         \
         } else {                                                                                             \
+            float e8_[8];                                                                                    \
+            (SUM) += exp_chunk<FEAT>(Z, s_hi, s_lo, (O), e8_, (SX));                                         \
             float4 *d_ = es + (size_t)((SLOT) * 4 + (ROWOFF)) * NCONS + tid;                                 \
             d_[0] = make_float4(e8_[0], e8_[1], e8_[2], e8_[3]);                                             \
             d_[NCONS] = make_float4(e8_[4], e8_[5], e8_[6], e8_[7]);                                         \
         }                                                                                                    \
+        if (FEAT) (BX) = fmaxf((BX), fmaf(zm_, s_lo, fmaf(zm_, s_hi, -(O))));                                \
     } while (0)
 
 // ------------------------------------------------------------------------------------------------
@@ -499,7 +502,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
             const bool hq = warp_has_children(parent, P.N, a, lane);
 
             // ---- pass 1: logits -> e, per-thread sums --------------------------------------------------
-            float ep[RT][8], eq[RT][8];
+            float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
             float op_f = 0.f, oq_f = 0.f;        // the thread's reference per row (integer-valued)
             bool set_p = false, set_q = false;
             float Sp_t = 0.f, Sq_t = 0.f, SXp_t = 0.f, SXq_t = 0.f;
@@ -508,37 +511,41 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
             {
                 RawChunk<DT> raw_p, raw_q;
                 float z[8];
+                float dummy[8];
                 for (int i = 0; i < nsm; ++i) {
                     SPECV_NEXT_TILE(i)
                     unpack_chunk<DT>(raw_p, z);
                     mask_chunk(z, nvalid, has_cut, cut_p);
-                    SPECV_P1_ROW(z, ep, 0, i, false, 0, i, 0, op_f, set_p, Sp_t, SXp_t, bxp);
+                    SPECV_P1_ROW(z, dummy, i, false, 0, i, , op_f, set_p, Sp_t, SXp_t, bxp);
                     if (hq) {
                         unpack_chunk<DT>(raw_q, z);
                         mask_chunk(z, nvalid, has_cut, cut_q);
-                        SPECV_P1_ROW(z, eq, 0, i, false, 2, i, 0, oq_f, set_q, Sq_t, SXq_t, bxq);
+                        SPECV_P1_ROW(z, dummy, i, false, 2, i, , oq_f, set_q, Sq_t, SXq_t, bxq);
                     }
                 }
-#pragma unroll
-                for (int j = 0; j < RT; ++j) {
-                    if (j < nrg) {
-                        SPECV_NEXT_TILE(nsm + j)
-                        unpack_chunk<DT>(raw_p, z);
-                        mask_chunk(z, nvalid, has_cut, cut_p);
-                        SPECV_P1_ROW(z, ep, j, 0, true, 0, nsm, j, op_f, set_p, Sp_t, SXp_t, bxp);
-                        if (hq) {
-                            unpack_chunk<DT>(raw_q, z);
-                            mask_chunk(z, nvalid, has_cut, cut_q);
-                            SPECV_P1_ROW(z, eq, j, 0, true, 2, nsm, j, oq_f, set_q, Sq_t, SXq_t, bxq);
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) eq[j][k] = 0.f;
-                        }
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) { ep[j][k] = 0.f; eq[j][k] = 0.f; }
-                    }
+// one register tile: J its number, EP / EQ its arrays, RP / RQ the statements rescaling the earlier ones
+#define SPECV_REG_TILE(J, EP, EQ, RP, RQ)                                                                    \
+                if ((J) < nrg) {                                                                             \
+                    SPECV_NEXT_TILE(nsm + (J))                                                               \
+                    unpack_chunk<DT>(raw_p, z);                                                              \
+                    mask_chunk(z, nvalid, has_cut, cut_p);                                                   \
+                    SPECV_P1_ROW(z, EP, 0, true, 0, nsm, RP, op_f, set_p, Sp_t, SXp_t, bxp);                 \
+                    if (hq) {                                                                                \
+                        unpack_chunk<DT>(raw_q, z);                                                          \
+                        mask_chunk(z, nvalid, has_cut, cut_q);                                               \
+                        SPECV_P1_ROW(z, EQ, 0, true, 2, nsm, RQ, oq_f, set_q, Sq_t, SXq_t, bxq);             \
+                    } else {                                                                                 \
+                        _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                           \
+                    }                                                                                        \
+                } else {                                                                                     \
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) { EP[k] = 0.f; EQ[k] = 0.f; }              \
                 }
+                SPECV_REG_TILE(0, ep0, eq0, , )
+                SPECV_REG_TILE(1, ep1, eq1, SPECV_SCALE8(ep0, f_);, SPECV_SCALE8(eq0, f_);)
+                SPECV_REG_TILE(2, ep2, eq2, SPECV_SCALE8(ep0, f_); SPECV_SCALE8(ep1, f_);, SPECV_SCALE8(eq0, f_); SPECV_SCALE8(eq1, f_);)
+                SPECV_REG_TILE(3, ep3, eq3, SPECV_SCALE8(ep0, f_); SPECV_SCALE8(ep1, f_); SPECV_SCALE8(ep2, f_);,
+                               SPECV_SCALE8(eq0, f_); SPECV_SCALE8(eq1, f_); SPECV_SCALE8(eq2, f_);)
+#undef SPECV_REG_TILE
             }
             const int op_t = set_p ? (int)op_f : OMIN, oq_t = set_q ? (int)oq_f : OMIN;
 
@@ -782,8 +789,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
                     load_e8(d + 2 * NCONS, NCONS, q);
                     tot += residual_chunk(p, q, g_hi, g_lo);
                 }
-#pragma unroll
-                for (int jr = 0; jr < RT; ++jr) tot += residual_chunk(ep[jr], eq[jr], g_hi, g_lo);
+                tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
+                       (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
                 const double wsum = W.A * warp_sum((double)(tot * phi_t));
                 const int par = xn & 1;
                 if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
@@ -857,10 +864,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
                     const double r = warp_sum((double)(residual_chunk(p, q, gh_c, gl_c) * phi_t));
                     if (lane == 0) S.wtile[warp][i] = r;
                 }
-#pragma unroll
-                for (int jr = 0; jr < RT; ++jr) {
-                    const double r = warp_sum((double)(residual_chunk(ep[jr], eq[jr], gh_c, gl_c) * phi_t));
-                    if (lane == 0) S.wtile[warp][nsm + jr] = r;
+                {
+                    const double r0 = warp_sum((double)(residual_chunk(ep0, eq0, gh_c, gl_c) * phi_t));
+                    const double r1 = warp_sum((double)(residual_chunk(ep1, eq1, gh_c, gl_c) * phi_t));
+                    const double r2 = warp_sum((double)(residual_chunk(ep2, eq2, gh_c, gl_c) * phi_t));
+                    const double r3 = warp_sum((double)(residual_chunk(ep3, eq3, gh_c, gl_c) * phi_t));
+                    if (lane == 0) {
+                        S.wtile[warp][nsm] = r0; S.wtile[warp][nsm + 1] = r1;
+                        S.wtile[warp][nsm + 2] = r2; S.wtile[warp][nsm + 3] = r3;
+                    }
                 }
                 bar_sync(1, NCONS);
                 // tile, then warp inside the tile, then lane inside the warp, then token inside the chunk
@@ -884,12 +896,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_verify_ke
                         load_e8(d, NCONS, p);
                         load_e8(d + 2 * NCONS, NCONS, q);
                     } else {
+                        const int jr = i_star - nsm;
 #pragma unroll
-                        for (int jr = 0; jr < RT; ++jr)
-                            if (jr == i_star - nsm) {
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) { p[k] = ep[jr][k]; q[k] = eq[jr][k]; }
-                            }
+                        for (int k = 0; k < 8; ++k) {
+                            p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
+                            q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
+                        }
                     }
                     float wk[8], v = 0.f;
 #pragma unroll
