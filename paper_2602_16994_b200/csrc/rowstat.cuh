@@ -17,6 +17,7 @@
 #pragma once
 #include "common.cuh"
 #include "cut.cuh"
+#include "stream.cuh"
 
 namespace specv {
 namespace rowstat {
@@ -27,17 +28,6 @@ constexpr int NB = cut::NB;
 constexpr int PER = NB / NT;
 constexpr int CMAXR = 16;
 
-struct __align__(16) RowStat {
-    double Z;          // sum over kept tokens of 2^(z s - O)
-    double X;          // sum over kept tokens of e x, x = z s - O (entropy = ln Z - ln2 X / Z)
-    int O;             // reference: ceil(max z s); OMIN-like sentinel when the row has no finite logit
-    float cut;         // smallest kept logit (-inf: nothing cut)
-    float xmax;        // largest exponent x (top-1 probability = 2^xmax / Z)
-    int kept;
-    int bad;           // 1: NaN / +inf in the row, or no finite logit
-    int pad;
-};
-
 struct RParams {
     int B, N, V, C, dtype, top_k;
     int slice_len;             // tokens per CTA slice (multiple of 8)
@@ -47,7 +37,7 @@ struct RParams {
     const int *parent;         // NULL: every row of `zp` only (spec_tree_probs)
     float T;
     const float *T_seq;
-    RowStat *stat;             // [B*N*2]
+    RowPart *part;             // [B*N*2]: the row's statistics as one slice
     float *cut;                // [B*N*2] (the verify kernel reads the cuts from here)
 };
 
@@ -259,7 +249,7 @@ __global__ void __launch_bounds__(NT, 2) spec_row_stat_kernel(const RParams P)
         const long long row = id >> 1;
         const int which = (int)(id & 1);
         const int b = (int)(row / P.N), a = (int)(row % P.N);
-        RowStat *out = P.stat + row * 2 + which;
+        RowPart *out = P.part + row * 2 + which;
         if (which == 1) {
             bool any = false;
             if (P.parent) {
@@ -268,8 +258,8 @@ __global__ void __launch_bounds__(NT, 2) spec_row_stat_kernel(const RParams P)
             }
             if (!__syncthreads_or((int)any)) {        // a draft row is read only for nodes with children
                 if (rank == 0 && tid == 0) {
-                    RowStat r = {};
-                    r.cut = -CUDART_INF_F; r.O = -(1 << 30);
+                    RowPart r = {};
+                    r.cut = -CUDART_INF_F; r.O = ROWPART_EMPTY; r.bad = -1;        // row not read
                     *out = r;
                     P.cut[row * 2 + 1] = -CUDART_INF_F;
                 }
@@ -483,10 +473,11 @@ __global__ void __launch_bounds__(NT, 2) spec_row_stat_kernel(const RParams P)
             for (int r = 0; r < C; ++r) { Z += S.xv[xpar][r][0]; X += S.xv[xpar][r][1]; K += S.xv[xpar][r][2]; }
             xpar ^= 1;
             if (rank == 0 && tid == 0) {
-                RowStat r;
-                r.Z = Z; r.X = X; r.O = bad ? -(1 << 30) : (int)of; r.cut = cutv;
+                RowPart r;
+                r.S = Z; r.X = X; r.O = bad ? ROWPART_EMPTY : (int)of; r.cut = cutv;
                 r.xmax = bad ? 0.f : (float)((double)m * s_d - (double)of);
-                r.kept = (int)K; r.bad = bad ? 1 : 0; r.pad = 0;
+                r.bad = bad ? 1 : 0;
+                (void)K;
                 *out = r;
                 P.cut[row * 2 + which] = cutv;
             }

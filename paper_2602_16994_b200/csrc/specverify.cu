@@ -16,6 +16,7 @@
 #include "rowstat.cuh"
 #include "specverify.h"
 #include "verify.cuh"
+#include "walk.cuh"
 
 namespace specv {
 namespace {
@@ -152,7 +153,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 struct WsLayout {
     int64_t rec, pub, done, cut, stat, clear_bytes, total;
 };
-WsLayout ws_layout(const SpecIn *in)
+WsLayout ws_layout(const SpecIn *in, int slices = 32)
 {
     WsLayout L;
     const int64_t nodes = (int64_t)in->B * in->N;
@@ -163,7 +164,7 @@ WsLayout ws_layout(const SpecIn *in)
     L.clear_bytes = o - L.pub;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
-    L.stat = o; o += up256(nodes * 2 * (int64_t)sizeof(rowstat::RowStat));
+    L.stat = o; o += up256(nodes * 2 * slices * (int64_t)sizeof(RowPart));      // row statistics, per slice
     L.total = o;
     return L;
 }
@@ -282,7 +283,7 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
     rp.top_k = in->top_k; rp.top_p = in->top_p; rp.slice_len = up((in->V + C - 1) / C, 8);
     rp.zp = zp; rp.zq = zq; rp.seq_stride = in->seq_stride; rp.node_stride = in->node_stride;
     rp.topo_stride = in->topo_seq_stride; rp.parent = parent; rp.T = in->temperature; rp.T_seq = in->temperature_per_seq;
-    rp.stat = (rowstat::RowStat *)(ws + L.stat); rp.cut = (float *)(ws + L.cut);
+    rp.part = (RowPart *)(ws + L.stat); rp.cut = (float *)(ws + L.cut);
     const int smem = up(rp.slice_len * esz, 128);
     const long long items = 2ll * in->B * in->N;
     int rc, nc;
@@ -302,7 +303,62 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
     return launch_clustered(k, nc * C, C, rowstat::NT, smem, st, &rp);
 }
 
-int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode)
+// SpecInfer without diagnostic outputs: row statistics of every row, then one walk per sequence
+template <int DT, int NW>
+int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
+{
+    auto kernel = spec_walk_kernel<DT, NW>;
+    int rc = prepare_kernel(kernel, pl.C, pl.smem);
+    if (rc) return rc;
+    const int threads = (NW + 1) * 32;
+    int nc = resident_clusters(kernel, pl.C, threads, pl.smem);
+    if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
+    if (nc > wp.B) nc = wp.B;
+    return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &wp);
+}
+
+int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl,
+                bool trunc, cudaStream_t st)
+{
+    int rc;
+    int NSL = 1;
+    RowPart *part = (RowPart *)(w + L.stat);
+    if (trunc) {
+        rc = launch_rowstat(in, in->target_logits, in->draft_logits, in->parent, w, L, st);
+        if (rc) return rc;
+    } else {
+        NSL = (in->V + stream::SLICE - 1) / stream::SLICE;
+        if (NSL > 32) return SPEC_ERR_UNSUPPORTED;
+        stream::SParams sp = {};
+        sp.B = in->B; sp.N = in->N; sp.V = in->V; sp.NSL = NSL;
+        sp.zp = in->target_logits; sp.zq = in->draft_logits;
+        sp.seq_stride = in->seq_stride; sp.node_stride = in->node_stride; sp.topo_stride = in->topo_seq_stride;
+        sp.parent = in->parent; sp.T = in->temperature; sp.T_seq = in->temperature_per_seq; sp.part = part;
+        const unsigned grid = (unsigned)(2ll * in->B * in->N * NSL);
+        if (in->logits_dtype == SPEC_BF16) stream::spec_row_partial_kernel<SPEC_BF16><<<grid, stream::NT, 0, st>>>(sp);
+        else stream::spec_row_partial_kernel<SPEC_F32><<<grid, stream::NT, 0, st>>>(sp);
+        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    }
+    if (out->node_features) {
+        stream::FParams fp = {(long long)in->B * in->N, NSL, part, out->node_features};
+        const unsigned grid = (unsigned)(((long long)in->B * in->N * 32 + 255) / 256);
+        stream::spec_features_kernel<<<grid, 256, 0, st>>>(fp);
+        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    }
+    WParams wp = {};
+    wp.B = in->B; wp.N = in->N; wp.V = in->V; wp.C = pl.C; wp.NSL = NSL;
+    wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.off_x = pl.off_x; wp.off_es = pl.off_es; wp.off_ring = pl.off_ring;
+    wp.zp = in->target_logits; wp.zq = in->draft_logits;
+    wp.seq_stride = in->seq_stride; wp.node_stride = in->node_stride; wp.topo_stride = in->topo_seq_stride;
+    wp.parent = in->parent; wp.token = in->token; wp.T = in->temperature; wp.T_seq = in->temperature_per_seq;
+    wp.part = part; wp.u_accept = in->u_accept; wp.u_bonus = in->u_bonus; wp.out = *out;
+    const bool bf = in->logits_dtype == SPEC_BF16;
+    if (pl.NW == 7) return bf ? launch_walk<SPEC_BF16, 7>(pl, wp, st) : launch_walk<SPEC_F32, 7>(pl, wp, st);
+    return bf ? launch_walk<SPEC_BF16, 15>(pl, wp, st) : launch_walk<SPEC_F32, 15>(pl, wp, st);
+}
+
+int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode,
+                  bool allow_walk = true)
 {
     int rc = check_in(in, true);
     if (rc) return rc;
@@ -315,6 +371,8 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     if (!make_vplan(in->V, in->logits_dtype, &pl)) return SPEC_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char *w = (unsigned char *)ws;
+    const bool diagnostics = out->residual || out->node_thr || out->node_w_in || out->margin;
+    if (allow_walk && mode == MODE_SPECINFER && !diagnostics) return verify_walk(in, out, w, L, pl, trunc, st);
     if (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
         cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess) {
         cudaGetLastError();
@@ -401,7 +459,7 @@ HostLayout host_layout(const SpecIn *in)
 // ------------------------------------------------------------------------------------------------
 // scratch that lives inside the library image, for spec_verify_specinfer_static
 // ------------------------------------------------------------------------------------------------
-constexpr int64_t STATIC_WS_BYTES = 640 * 1024;
+constexpr int64_t STATIC_WS_BYTES = 1024 * 1024;
 static __device__ __align__(256) unsigned char g_static_ws[STATIC_WS_BYTES];
 
 // Device address of g_static_ws on the current device.  In host code the array's name is only a
@@ -466,11 +524,11 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
 {
     int rc = check_in(in, true);
     if (rc) return rc;
-    if ((int64_t)in->B * in->N > SPEC_STATIC_MAX_NODES || ws_layout(in).total > STATIC_WS_BYTES) return SPEC_ERR_WORKSPACE;
+    if ((int64_t)in->B * in->N > SPEC_STATIC_MAX_NODES || ws_layout(in, 1).total > STATIC_WS_BYTES) return SPEC_ERR_WORKSPACE;
     void *ws = nullptr;
     rc = static_ws_address(&ws);
     if (rc) return rc;
-    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER);
+    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false);
 }
 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,

@@ -1,0 +1,521 @@
+// SpecInfer verification as a walk (Algorithm 4 composed top-down, Section 3.2), one thread-block
+// cluster per sequence, on top of the row statistics (stream.cuh / rowstat.cuh).
+//
+// With every row's normaliser known, the decision about a node's FIRST child needs no vocabulary-wide
+// work: its threshold is min(1, p(x)/q(x)), two logits and two normalisers.  The cluster therefore walks
+// down the tree with scalar arithmetic only, and brings a node's rows on chip (the same machinery as
+// the fused kernel: producer warp + bulk-copy ring, e = 2^(z s - O) resident in registers and shared
+// memory, one pass + one distributed-shared-memory exchange per sibling step, inverse-CDF search) only
+// where Algorithm 4 needs a residual: at a node whose first child was rejected, and at the stop node
+// for the bonus draw.  That is one or two resident nodes per sequence instead of every node of the tree.
+//
+// Every consumer warp of the cluster runs the same walk on the same numbers (the exchanges deliver
+// bit-identical totals to all of them), so control flow agrees across the cluster without barriers.
+// The thread that finds the bonus token writes all outputs of the sequence.
+#pragma once
+#include "stream.cuh"
+#include "verify.cuh"
+
+namespace specv {
+
+struct WParams {
+    int B, N, V, C, NSL;
+    int slice_len, NS, off_x, off_es, off_ring;
+    const void *zp, *zq;
+    long long seq_stride, node_stride, topo_stride;
+    const int *parent, *token;
+    float T;
+    const float *T_seq;
+    const RowPart *part;      // [B*N*2][NSL]
+    const float *u_accept, *u_bonus;
+    SpecOut out;
+};
+
+struct __align__(16) WHdr {
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], req, ack;
+    double wtile[NWMAX + 1][TMAX];
+    WarpArea wa[NWMAX];
+    int req_a, req_b, req_hq;
+    int poison;
+};
+
+// merged statistics of one row: reference, normaliser, cut, entropy sum, largest exponent, validity
+struct RowSum {
+    double Z, X;
+    int O;
+    float cut, xmax;
+    int bad;        // 1: NaN / +inf / no finite logit
+};
+
+// every lane gets the same answer; lanes share the slices of the row
+__device__ __forceinline__ RowSum merge_row(const RowPart *part, long long row2, int NSL, int lane)
+{
+    int O = ROWPART_EMPTY, bad = 0;
+    float cutv = -CUDART_INF_F;
+    for (int j = lane; j < NSL; j += 32) {
+        const RowPart *p = part + row2 * NSL + j;
+        O = max(O, __ldcg(&p->O));
+        bad |= __ldcg(&p->bad) == 1;
+        if (j == 0) cutv = __ldcg(&p->cut);
+    }
+    O = __reduce_max_sync(0xffffffffu, O);
+    double S = 0.0, X = 0.0, best = -1.0e300;
+    for (int j = lane; j < NSL; j += 32) {
+        const RowPart *p = part + row2 * NSL + j;
+        const int o = __ldcg(&p->O);
+        if (o > ROWPART_EMPTY) {
+            const int d = max(o - O, -100000);
+            const double f = pow2d(d), s = __ldcg(&p->S);
+            S += s * f;
+            X += f * (__ldcg(&p->X) + (double)d * s);
+            best = fmax(best, (double)o + (double)__ldcg(&p->xmax));
+        }
+    }
+    RowSum r;
+    r.Z = warp_sum(S);
+    r.X = warp_sum(X);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
+    r.O = O;
+    r.cut = __shfl_sync(0xffffffffu, cutv, 0);
+    r.xmax = O > ROWPART_EMPTY ? (float)(best - (double)O) : 0.f;
+    r.bad = __any_sync(0xffffffffu, bad) || !(r.Z > 0.0) || !(r.Z < CUDART_INF);
+    return r;
+}
+
+template <int DT, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kernel(const WParams P)
+{
+    constexpr bool FEAT = false;
+    constexpr int NCONS = NW * 32;
+    constexpr int TILE = NCONS * 8;
+    constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
+    constexpr int ROWB = TILE * ESZ;
+    constexpr int STAGE = 2 * ROWB;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    WHdr &S = *reinterpret_cast<WHdr *>(dyn_smem);
+    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW]
+    float4 *es = reinterpret_cast<float4 *>(dyn_smem + P.off_es);    // [slot][p lo, p hi, q lo, q hi][NCONS]
+    unsigned char *ring = dyn_smem + P.off_ring;
+    const int C = P.C, NS = P.NS;
+    const unsigned rank = cluster_ctarank();
+    const int cid = blockIdx.x / C, NC = gridDim.x / C;
+    const long long tok0 = (long long)rank * P.slice_len;
+    const int n_slice = (int)max(0ll, min((long long)P.slice_len, (long long)P.V - tok0));
+    const int ntiles = (n_slice + TILE - 1) / TILE;
+    const int nsm = max(ntiles - RT, 0), nrg = ntiles - nsm;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], NW); }
+        mbar_init(&S.xbar[0], 1);
+        mbar_init(&S.xbar[1], 1);
+        mbar_init(&S.req, 1);
+        mbar_init(&S.ack, 1);
+        S.poison = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    cluster_sync_all();
+
+    if (warp == NW) {
+        // ======================= producer warp: loads the node the consumers ask for =====================
+        int g = 0;
+        uint32_t rphase = 0;
+        for (;;) {
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(&S.req, rphase) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            rphase ^= 1u;
+            if (!ok) { S.poison = 1; break; }
+            const int a = *(volatile int *)&S.req_a, b = *(volatile int *)&S.req_b;
+            const bool hq = *(volatile int *)&S.req_hq != 0;
+            if (lane == 0) mbar_arrive(&S.ack);          // the request has been read: the next one may be posted
+            if (a < 0) break;
+            const long long row = (long long)b * P.seq_stride + (long long)a * P.node_stride + tok0;
+            const unsigned char *src_p = (const unsigned char *)P.zp + row * ESZ;
+            const unsigned char *src_q = (const unsigned char *)P.zq + row * ESZ;
+            const bool aligned = ((((uintptr_t)src_p) | (hq ? (uintptr_t)src_q : 0)) & 15) == 0;
+            bool fail = false;
+            for (int i = 0; i < ntiles; ++i, ++g) {
+                const int stage = g % NS, use = g / NS;
+                if (use > 0) {
+                    int w = 1;
+                    if (lane == 0) w = mbar_wait(&S.empty[stage], (uint32_t)((use - 1) & 1)) ? 1 : 0;
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w || *(volatile int *)&S.poison) { S.poison = 1; fail = true; break; }
+                }
+                const int ntok = min(TILE, n_slice - i * TILE);
+                unsigned char *dst_p = ring + (size_t)stage * STAGE, *dst_q = dst_p + ROWB;
+                const unsigned char *sp = src_p + (size_t)i * ROWB, *sq = src_q + (size_t)i * ROWB;
+                const uint32_t body = aligned ? (((uint32_t)ntok * ESZ) & ~15u) : 0u;
+                if (ESZ == 2) {
+                    for (int e = (int)(body / 2) + lane; e < ntok; e += 32) {
+                        ((unsigned short *)dst_p)[e] = __ldg((const unsigned short *)sp + e);
+                        if (hq) ((unsigned short *)dst_q)[e] = __ldg((const unsigned short *)sq + e);
+                    }
+                } else {
+                    for (int e = (int)(body / 4) + lane; e < ntok; e += 32) {
+                        ((float *)dst_p)[e] = __ldg((const float *)sp + e);
+                        if (hq) ((float *)dst_q)[e] = __ldg((const float *)sq + e);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    if (body) {
+                        mbar_arrive_expect_tx(&S.full[stage], hq ? 2 * body : body);
+                        bulk_g2s(dst_p, sp, body, &S.full[stage]);
+                        if (hq) bulk_g2s(dst_q, sq, body, &S.full[stage]);
+                    } else {
+                        mbar_arrive(&S.full[stage]);
+                    }
+                }
+            }
+            if (fail) {
+                if (lane == 0)
+                    for (int k = 1; k <= NS && k <= g; ++k) {
+                        const int gg = g - k;
+                        mbar_wait(&S.full[gg % NS], (uint32_t)((gg / NS) & 1));
+                    }
+                break;
+            }
+        }
+    } else {
+        // ================================ consumer warps: the walk ==========================================
+        WarpArea &W = S.wa[warp];
+        int stage = 0;
+        uint32_t phase = 0;
+        int xn = 0;
+        uint32_t aphase = 0;        // warp 0, lane 0: requests acknowledged so far (parity)
+        bool posted = false;
+        float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
+
+        for (int b = cid; b < P.B; b += NC) {
+            const int *parent = P.parent + (long long)b * P.topo_stride;
+            const int *token = P.token + (long long)b * P.N;
+            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+            float s_hi = (float)s_d;
+            if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
+            float s_lo = (float)(s_d - (double)s_hi);
+            if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
+
+            // ---- the whole tree is checked first: topology, tokens, rows that are not finite ------------------
+            int status = 0;
+            for (int i = lane; i < P.N; i += 32) {
+                const int pa = __ldg(parent + i);
+                if (i == 0 ? (pa != -1) : (pa < 0 || pa >= i)) status = max(status, SPEC_DEV_TOPOLOGY);
+                if (i > 0) {
+                    const int x = __ldg(token + i);
+                    if (x < 0 || x >= P.V) status = max(status, SPEC_DEV_TOKEN);
+                }
+            }
+            {
+                // a row is not finite if a slice saw NaN / +inf, or if no slice has a finite logit
+                const long long rows2 = 2ll * P.N;
+                for (long long r2 = lane; r2 < rows2; r2 += 32) {
+                    const RowPart *p = P.part + ((long long)b * rows2 + r2) * P.NSL;
+                    int any_finite = 0, bad = 0, unread = 0;
+                    for (int j = 0; j < P.NSL; ++j) {
+                        const int bd = __ldcg(&p[j].bad);
+                        unread |= bd == -1;
+                        bad |= bd == 1;
+                        any_finite |= __ldcg(&p[j].O) > ROWPART_EMPTY && __ldcg(&p[j].S) > 0.0;
+                    }
+                    if (!unread && (bad || !any_finite)) status = max(status, SPEC_DEV_NONFINITE);
+                }
+            }
+            status = __reduce_max_sync(0xffffffffu, status);
+            int cur = 0, len = 0;
+            int bonus = -1;
+            bool writer = false;          // this lane writes the sequence's outputs
+            bool done = status != 0;
+            if (done && rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
+
+            while (!done) {
+                const int a = cur;
+                // ---- children of a ------------------------------------------------------------------------------
+                int kc = 0;
+                for (int c0 = a + 1; c0 < P.N; c0 += 32) {
+                    const int c = c0 + lane;
+                    const bool is = c < P.N && __ldg(parent + c) == a;
+                    const unsigned bal = __ballot_sync(0xffffffffu, is);
+                    if (is) {
+                        const int pos = kc + __popc(bal & ((1u << lane) - 1u));
+                        if (pos < KMAX) {
+                            W.child[pos] = c;
+                            W.cpn[pos] = __ldg(token + c);
+                            W.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
+                        }
+                    }
+                    kc += __popc(bal);
+                }
+                if (kc > KMAX) { status = SPEC_DEV_TOPOLOGY; done = true; if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; } break; }
+                const bool hq = kc > 0;
+                const RowSum rp = merge_row(P.part, ((long long)b * P.N + a) * 2, P.NSL, lane);
+                RowSum rq = rp;
+                if (hq) rq = merge_row(P.part, ((long long)b * P.N + a) * 2 + 1, P.NSL, lane);
+                const double invZp = __drcp_rn(rp.Z), invZq = hq ? __drcp_rn(rq.Z) : 0.0;
+                // target / draft probability of every child's token (lanes j and 16 + j)
+                __syncwarp();
+                {
+                    const int j = lane & 15;
+                    const bool mine = j < kc;
+                    const int xt = mine ? W.cpn[j] : 0;
+                    __syncwarp();
+                    if (mine) {
+                        const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
+                        const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + xt);
+                        const double xd = (double)z * s_d - (double)(lane < 16 ? rp.O : rq.O);
+                        double pr = 0.0;
+                        if (z >= (lane < 16 ? rp.cut : rq.cut) && xd > -1000.0) {
+                            const double nd = rint(xd);
+                            pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
+                        }
+                        if (lane < 16) W.cpm[j] = pr; else W.cqm[j] = pr;
+                    }
+                    __syncwarp();
+                }
+                // ---- first child: needs no residual -------------------------------------------------------------------
+                bool resident = false;
+                double st_c = 0.0, st_E = 1.0, g_commit = 0.0;
+                double E_r = 0.0;
+                int acc = -1;
+                int j0 = 0;
+                if (hq) {
+                    const double Pp = W.cpm[0], Pq = W.cqm[0];
+                    const bool zero = !(Pp > 0.0), one = !zero && !(Pq > 0.0);
+                    if (!zero && (one || (double)W.cu[0] * Pq < Pp)) acc = W.child[0];
+                    j0 = 1;
+                }
+                if (acc < 0) {
+                    // ---- the node comes on chip: e = 2^(z s - O) of both rows ----------------------------------------
+                    resident = true;
+                    if (warp == 0 && lane == 0) {
+                        if (posted) { if (!mbar_wait(&S.ack, aphase)) S.poison = 1; aphase ^= 1u; }
+                        S.req_a = a; S.req_b = b; S.req_hq = hq ? 1 : 0;
+                        mbar_arrive(&S.req);
+                        posted = true;
+                    }
+                    bool poisoned = *(volatile int *)&S.poison != 0;
+                    const float ofp = (float)rp.O, ofq = (float)rq.O;
+                    {
+                        RawChunk<DT> raw_p, raw_q;
+                        float z[8];
+                        float dsx = 0.f;
+#define SPECW_NEXT_TILE(TILE_INDEX)                                                                          \
+                        if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; } \
+                        {                                                                                    \
+                            const unsigned char *sp_ = ring + (size_t)stage * STAGE + (size_t)tid * 8 * ESZ; \
+                            raw_p = read_raw<DT>(sp_);                                                       \
+                            if (hq) raw_q = read_raw<DT>(sp_ + ROWB);                                        \
+                        }                                                                                    \
+                        __syncwarp();                                                                        \
+                        if (lane == 0) mbar_arrive(&S.empty[stage]);                                         \
+                        if (++stage == NS) { stage = 0; phase ^= 1u; }                                       \
+                        const int nvalid = poisoned ? 0 : n_slice - ((TILE_INDEX) * TILE + tid * 8);
+                        for (int i = 0; i < nsm; ++i) {
+                            SPECW_NEXT_TILE(i)
+                            float e8[8];
+                            unpack_chunk<DT>(raw_p, z);
+                            mask_chunk(z, nvalid, true, rp.cut);
+                            exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
+                            float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                            d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
+                            d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
+                            if (hq) {
+                                unpack_chunk<DT>(raw_q, z);
+                                mask_chunk(z, nvalid, true, rq.cut);
+                                exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
+                                d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
+                                d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
+                            } else {
+                                d[2 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                d[3 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+                        }
+#define SPECW_REG_TILE(J, EP, EQ)                                                                            \
+                        if ((J) < nrg) {                                                                     \
+                            SPECW_NEXT_TILE(nsm + (J))                                                       \
+                            unpack_chunk<DT>(raw_p, z);                                                      \
+                            mask_chunk(z, nvalid, true, rp.cut);                                             \
+                            exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                    \
+                            if (hq) {                                                                        \
+                                unpack_chunk<DT>(raw_q, z);                                                  \
+                                mask_chunk(z, nvalid, true, rq.cut);                                         \
+                                exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                \
+                            } else {                                                                         \
+                                _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                   \
+                            }                                                                                \
+                        } else {                                                                             \
+                            _Pragma("unroll") for (int k = 0; k < 8; ++k) { EP[k] = 0.f; EQ[k] = 0.f; }      \
+                        }
+                        SPECW_REG_TILE(0, ep0, eq0)
+                        SPECW_REG_TILE(1, ep1, eq1)
+                        SPECW_REG_TILE(2, ep2, eq2)
+                        SPECW_REG_TILE(3, ep3, eq3)
+#undef SPECW_REG_TILE
+#undef SPECW_NEXT_TILE
+                    }
+                    // ---- sibling steps (the first child, if any, is already rejected) ------------------------------------
+                    const double Rg = hq ? rp.Z * invZq : 0.0;          // pass coefficient g = c Rg (w_in = 1, G = E)
+                    int j = j0;
+                    for (;;) {
+                        // one pass + exchange with the coefficient of the current state: c = st_c + (rejections so far)
+                        const double cnext = (hq && j > 0) ? st_c + st_E : 0.0;
+                        const double g = cnext * Rg;
+                        float g_hi, g_lo;
+                        split_float(g, g_hi, g_lo);
+                        float tot = 0.f;
+                        for (int i = 0; i < nsm; ++i) {
+                            float p[8], q[8];
+                            const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                            load_e8(d, NCONS, p);
+                            load_e8(d + 2 * NCONS, NCONS, q);
+                            tot += residual_chunk(p, q, g_hi, g_lo);
+                        }
+                        tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
+                               (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
+                        const double wsum = invZp * warp_sum((double)tot);
+                        const int par = xn & 1;
+                        if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
+                        if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
+                        if (!*(volatile int *)&S.poison && !mbar_wait_cluster(&S.xbar[par], (uint32_t)((xn >> 1) & 1))) S.poison = 1;
+                        ++xn;
+                        double y = 0.0;
+                        if (lane < C) {
+                            const double *src = xchg + (size_t)(par * C + lane) * NW;
+#pragma unroll
+                            for (int w = 0; w < NW; ++w) y += src[w];
+                        }
+                        const double En = warp_sum(y);
+                        if (*(volatile int *)&S.poison) { status = SPEC_DEV_TIMEOUT; break; }
+                        if (En > 0.0 || j == 0) {
+                            if (j > 0) { st_c = cnext; }
+                            st_E = j > 0 ? En : 1.0;
+                            g_commit = g;
+                            E_r = y;
+                        }
+                        // else S = 0 with P equal to q up to rounding: the state stays
+                        if (j >= kc) break;
+                        // child j from the committed state
+                        const double Pp = W.cpm[j], Pq = W.cqm[j];
+                        const double Ux = Pp - st_c * Pq;
+                        const bool zero = !(Ux > 0.0), one = !zero && !(Pq > 0.0);
+                        if (!zero && (one || (double)W.cu[j] * st_E * Pq < Ux)) { acc = W.child[j]; break; }
+                        ++j;
+                    }
+                    if (status) { done = true; if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; } break; }
+                }
+                if (acc >= 0) { cur = acc; ++len; continue; }
+
+                // ---- stop here: the bonus token from the committed residual ---------------------------------------------
+                done = true;
+                const double E_tot = warp_sum(lane < C ? E_r : 0.0);
+                const double target = (double)__ldg(P.u_bonus + (long long)b * P.N + a) * E_tot;
+                double tau;
+                const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
+                if (owner < 0) {
+                    status = SPEC_DEV_NONFINITE;
+                    if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
+                } else if (owner == (int)rank) {
+                    float gh_c, gl_c;
+                    split_float(g_commit, gh_c, gl_c);
+                    const double tau_rel = tau * rp.Z, tot_rel = E_tot * rp.Z;      // in units of e
+                    for (int i = 0; i < nsm; ++i) {
+                        float p[8], q[8];
+                        const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                        load_e8(d, NCONS, p);
+                        load_e8(d + 2 * NCONS, NCONS, q);
+                        const double r = warp_sum((double)residual_chunk(p, q, gh_c, gl_c));
+                        if (lane == 0) S.wtile[warp][i] = r;
+                    }
+                    {
+                        const double r0 = warp_sum((double)residual_chunk(ep0, eq0, gh_c, gl_c));
+                        const double r1 = warp_sum((double)residual_chunk(ep1, eq1, gh_c, gl_c));
+                        const double r2 = warp_sum((double)residual_chunk(ep2, eq2, gh_c, gl_c));
+                        const double r3 = warp_sum((double)residual_chunk(ep3, eq3, gh_c, gl_c));
+                        if (lane == 0) {
+                            S.wtile[warp][nsm] = r0; S.wtile[warp][nsm + 1] = r1;
+                            S.wtile[warp][nsm + 2] = r2; S.wtile[warp][nsm + 3] = r3;
+                        }
+                    }
+                    bar_sync(1, NCONS);
+                    double Ti = 0.0;
+                    if (lane < nsm + RT)
+                        for (int w = 0; w < NW; ++w) Ti += S.wtile[w][lane];
+                    double tau2, tau3, tau4;
+                    const int i_star = pick_lane(Ti, tau_rel, tau2);
+                    const double Ww = (i_star >= 0 && lane < NW) ? S.wtile[lane][i_star] : 0.0;
+                    const int w_star = i_star >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
+                    bar_sync(1, NCONS);
+                    if (w_star < 0) {
+                        status = SPEC_DEV_NONFINITE;
+                        if (warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
+                    } else if (warp == w_star) {
+                        float p[8], q[8];
+                        if (i_star < nsm) {
+                            const float4 *d = es + (size_t)(i_star * 4) * NCONS + tid;
+                            load_e8(d, NCONS, p);
+                            load_e8(d + 2 * NCONS, NCONS, q);
+                        } else {
+                            const int jr = i_star - nsm;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
+                                q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
+                            }
+                        }
+                        float wk[8], v = 0.f;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl_c, q[k], fmaf(-gh_c, q[k], p[k])), 0.f); v += wk[k]; }
+                        const int l_star = pick_lane((double)v, tau3, tau4);
+                        if (l_star < 0) {
+                            status = SPEC_DEV_NONFINITE;
+                            if (lane == 0) { writer = true; cur = -1; len = -1; }
+                        } else if (lane == l_star) {
+                            double run = 0.0;
+                            int found = -1, last_pos = -1;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                run += (double)wk[k];
+                                if (wk[k] > 0.f) last_pos = k;
+                                if (found < 0 && run > tau4) found = k;
+                            }
+                            if (found < 0) found = last_pos;
+                            bonus = found >= 0 ? (int)(tok0 + (long long)i_star * TILE + tid * 8 + found) : -1;
+                            writer = true;
+                            if (bonus < 0) { status = SPEC_DEV_NONFINITE; cur = -1; len = -1; }
+                            (void)tot_rel;
+                        }
+                    }
+                }
+            }
+
+            // ---- outputs of the sequence (one thread) -----------------------------------------------------------------------
+            if (writer) {
+                const int st = status;
+                const int accn = st ? -1 : cur, ln = st ? -1 : len, bn = st ? -1 : bonus;
+                P.out.accepted_node[b] = accn;
+                P.out.accept_len[b] = ln;
+                P.out.bonus_token[b] = bn;
+                P.out.status[b] = st;
+                int *ot = P.out.out_tokens + (long long)b * P.N;
+                for (int i = 0; i < P.N; ++i) ot[i] = -1;
+                if (accn >= 0) {
+                    ot[ln] = bn;
+                    int i = ln;
+                    for (int x = accn; x != 0 && i > 0; x = __ldg(parent + x)) ot[--i] = __ldg(token + x);
+                }
+            }
+        }
+        // tell the producer to leave
+        if (warp == 0 && lane == 0) {
+            if (posted) { if (!mbar_wait(&S.ack, aphase)) S.poison = 1; aphase ^= 1u; }
+            S.req_a = -1;
+            mbar_arrive(&S.req);
+        }
+    }
+    __syncthreads();
+    cluster_sync_all();
+}
+
+}  // namespace specv
