@@ -153,7 +153,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 struct WsLayout {
     int64_t rec, pub, done, cut, stat, clear_bytes, total;
 };
-WsLayout ws_layout(const SpecIn *in, int slices = 32)
+WsLayout ws_layout(const SpecIn *in, int slices = 32)   // slices = 0: merged rows only
 {
     WsLayout L;
     const int64_t nodes = (int64_t)in->B * in->N;
@@ -164,7 +164,7 @@ WsLayout ws_layout(const SpecIn *in, int slices = 32)
     L.clear_bytes = o - L.pub;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
-    L.stat = o; o += up256(nodes * 2 * slices * (int64_t)sizeof(RowPart));      // row statistics, per slice
+    L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // merged rows, then slices
     L.total = o;
     return L;
 }
@@ -191,6 +191,19 @@ int launch_clustered(K kernel, int ctas, int C, int threads, int smem, cudaStrea
 }
 
 std::mutex g_cache_mutex;
+
+int sm_count()
+{
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 148; }
+    if (!cached[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { cudaGetLastError(); n = 148; }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
 
 // Kernel attributes are set once per (device, kernel): the largest dynamic shared memory asked for
 // so far and the permission for clusters above 8 CTAs.  Later calls only launch.
@@ -327,17 +340,31 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         rc = launch_rowstat(in, in->target_logits, in->draft_logits, in->parent, w, L, st);
         if (rc) return rc;
     } else {
-        NSL = (in->V + stream::SLICE - 1) / stream::SLICE;
-        if (NSL > 32) return SPEC_ERR_UNSUPPORTED;
+        // rows are split into parts only when there are fewer rows than resident CTAs
+        const long long rows2 = 2ll * in->B * in->N;
+        const int slices_row = (in->V + stream::SLICE - 1) / stream::SLICE;
+        NSL = 1;
+        while (NSL < 4 && NSL < slices_row && rows2 * NSL < 2 * sm_count()) NSL *= 2;
         stream::SParams sp = {};
         sp.B = in->B; sp.N = in->N; sp.V = in->V; sp.NSL = NSL;
         sp.zp = in->target_logits; sp.zq = in->draft_logits;
         sp.seq_stride = in->seq_stride; sp.node_stride = in->node_stride; sp.topo_stride = in->topo_seq_stride;
         sp.parent = in->parent; sp.T = in->temperature; sp.T_seq = in->temperature_per_seq; sp.part = part;
-        const unsigned grid = (unsigned)(2ll * in->B * in->N * NSL);
+        // parts go to the second half of the statistics region, the merged rows to its start; a row
+        // in one part is final as written.  One CTA per item: those of unread rows retire at once.
+        RowPart *parts = part + 2ll * in->B * in->N;
+        sp.part = NSL > 1 ? parts : part;
+        const long long items = 2ll * in->B * in->N * NSL;
+        const unsigned grid = (unsigned)(items < (1ll << 20) ? items : (1ll << 20));
         if (in->logits_dtype == SPEC_BF16) stream::spec_row_partial_kernel<SPEC_BF16><<<grid, stream::NT, 0, st>>>(sp);
         else stream::spec_row_partial_kernel<SPEC_F32><<<grid, stream::NT, 0, st>>>(sp);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+        if (NSL > 1) {
+            stream::MParams mp = {2ll * in->B * in->N, NSL, parts, part};
+            stream::spec_row_merge_kernel<<<(unsigned)((mp.rows2 * 32 + 255) / 256), 256, 0, st>>>(mp);
+            if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+        }
+        NSL = 1;
     }
     if (out->node_features) {
         stream::FParams fp = {(long long)in->B * in->N, NSL, part, out->node_features};
@@ -524,7 +551,7 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
 {
     int rc = check_in(in, true);
     if (rc) return rc;
-    if ((int64_t)in->B * in->N > SPEC_STATIC_MAX_NODES || ws_layout(in, 1).total > STATIC_WS_BYTES) return SPEC_ERR_WORKSPACE;
+    if ((int64_t)in->B * in->N > SPEC_STATIC_MAX_NODES || ws_layout(in, 0).total > STATIC_WS_BYTES) return SPEC_ERR_WORKSPACE;
     void *ws = nullptr;
     rc = static_ws_address(&ws);
     if (rc) return rc;

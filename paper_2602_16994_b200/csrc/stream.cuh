@@ -1,7 +1,7 @@
 // Streaming row statistics (no truncation): every logit row the verifiers may touch is read once from
 // HBM, straight into registers, and reduced to per-slice partial sums of the row's softmax normaliser.
-// No residency, no clusters: one CTA per (row, slice of 8192 tokens), 32 logits per thread loaded with
-// four 16-byte loads before any arithmetic, so a whole SM keeps more than 100 KB of loads in flight.
+// No residency, no clusters: a CTA streams a row (or a part of it) in slices of 8192 logits, 32 per thread,
+// the 16-byte loads of the next slice in flight while the current one is exponentiated.
 //
 // A thread turns its logits into e = 2^(z s - o) (s = log2(e)/T, o = ceil of its own largest z s, an
 // integer, so partial sums combine by exact powers of two) and the CTA writes, for its slice,
@@ -30,7 +30,7 @@ constexpr int PER = 32;                  // logits per thread
 constexpr int SLICE = NT * PER;          // logits per CTA
 
 struct SParams {
-    int B, N, V, NSL;
+    int B, N, V, NSL;        // NSL: parts a row is split into (more CTAs than rows)
     const void *zp, *zq;
     long long seq_stride, node_stride, topo_stride;
     const int *parent;
@@ -39,113 +39,220 @@ struct SParams {
     RowPart *part;           // [B*N*2][NSL]
 };
 
+// raw logits of one thread for one slice: PER / 8 chunks of 8
 template <int DT>
-__global__ void __launch_bounds__(NT, 4) spec_row_partial_kernel(const SParams P)
+struct RawItem {
+    uint4 v[DT == SPEC_BF16 ? PER / 8 : PER / 4];
+};
+
+// One CTA per (row, part of the row): the part's slices of 8192 logits are streamed one after the other,
+// the loads of the next slice issued before the arithmetic of the current one; each thread keeps a
+// running (reference, sum) pair, rescaled by an exact power of two when a later slice raises its
+// reference, and the CTA reduces once per part.
+template <int DT>
+__global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P)
 {
     constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
+    constexpr int NV = DT == SPEC_BF16 ? 1 : 2;           // 16-byte loads per chunk of 8 logits
     __shared__ double sS[NT / 32], sX[NT / 32], sB[NT / 32];
     __shared__ int sO[NT / 32], sBad[NT / 32];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const long long id = blockIdx.x;
-    const int j = (int)(id % P.NSL);
-    const long long row2 = id / P.NSL;
-    const int which = (int)(row2 & 1);
-    const long long row = row2 >> 1;
-    const int b = (int)(row / P.N), a = (int)(row % P.N);
-    RowPart *out = P.part + row2 * P.NSL + j;
-    if (which == 1) {
-        // a draft row is read only for nodes that have children
-        const int *parent = P.parent + (long long)b * P.topo_stride;
-        bool any = false;
-        for (int c = a + 1 + tid; c < P.N; c += NT) any |= __ldg(parent + c) == a;
-        if (!__syncthreads_or((int)any)) {
-            if (tid == 0) { RowPart r = {}; r.O = ROWPART_EMPTY; r.cut = -CUDART_INF_F; r.bad = -1; *out = r; }
-            return;
-        }
-    }
-    const int tok0 = j * SLICE;
-    const int n = min(SLICE, P.V - tok0);
-    const unsigned char *src = (const unsigned char *)(which ? P.zq : P.zp) +
-                               ((long long)b * P.seq_stride + (long long)a * P.node_stride + tok0) * ESZ;
-    const bool aligned = (((uintptr_t)src) & 15) == 0;
+    const long long items = 2ll * P.B * P.N * P.NSL;
+    const int slices_row = (P.V + SLICE - 1) / SLICE;
+    const int slices_part = (slices_row + P.NSL - 1) / P.NSL;
 
-    // ---- 32 logits per thread: chunk c of the thread is tokens (tid + c NT) * 8 ... + 8 -----------------------
-    float z[PER];
-#pragma unroll
-    for (int c = 0; c < PER / 8; ++c) {
-        const int t0 = (tid + c * NT) * 8;
-        if (aligned && t0 + 8 <= n) {
-            if (DT == SPEC_BF16) {
-                const uint4 r = __ldg(reinterpret_cast<const uint4 *>(src) + (tid + c * NT));
-                z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
-                z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
-            } else {
-                const float4 r0 = __ldg(reinterpret_cast<const float4 *>(src) + 2 * (tid + c * NT));
-                const float4 r1 = __ldg(reinterpret_cast<const float4 *>(src) + 2 * (tid + c * NT) + 1);
-                z[c * 8 + 0] = r0.x; z[c * 8 + 1] = r0.y; z[c * 8 + 2] = r0.z; z[c * 8 + 3] = r0.w;
-                z[c * 8 + 4] = r1.x; z[c * 8 + 5] = r1.y; z[c * 8 + 6] = r1.z; z[c * 8 + 7] = r1.w;
+    for (long long id = blockIdx.x; id < items; id += gridDim.x) {
+        const int h = (int)(id % P.NSL);
+        const long long row2 = id / P.NSL;
+        const int which = (int)(row2 & 1);
+        const long long row = row2 >> 1;
+        const int b = (int)(row / P.N), a = (int)(row % P.N);
+        RowPart *out = P.part + row2 * P.NSL + h;
+        if (which == 1) {
+            // a draft row is read only for nodes that have children
+            const int *parent = P.parent + (long long)b * P.topo_stride;
+            bool any = false;
+            for (int c = a + 1 + tid; c < P.N; c += NT) any |= __ldg(parent + c) == a;
+            if (!__syncthreads_or((int)any)) {
+                if (tid == 0) { RowPart r = {}; r.O = ROWPART_EMPTY; r.cut = -CUDART_INF_F; r.bad = -1; *out = r; }
+                continue;
             }
-        } else {
+        }
+        const unsigned char *rowp = (const unsigned char *)(which ? P.zq : P.zp) +
+                                    ((long long)b * P.seq_stride + (long long)a * P.node_stride) * ESZ;
+        const bool aligned = (((uintptr_t)rowp) & 15) == 0;
+        const int s_begin = h * slices_part, s_end = min(slices_row, s_begin + slices_part);
+        const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+        float s_hi = (float)s_d;
+        if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
+        float s_lo = (float)(s_d - (double)s_hi);
+        if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
+
+        // the thread's running state
+        float of = 0.f, S_t = 0.f, X_t = 0.f, xm_t = -CUDART_INF_F;
+        bool set = false;
+        int bad = 0;
+
+        RawItem<DT> nxt;
+        bool nxt_fast = false;
+        auto issue = [&](int sl, RawItem<DT> &r) -> bool {
+            if (sl >= s_end) return false;
+            const int n = min(SLICE, P.V - sl * SLICE);
+            if (!aligned || n < SLICE) return false;
+            const uint4 *src = reinterpret_cast<const uint4 *>(rowp + (size_t)sl * SLICE * ESZ);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
+            for (int c = 0; c < PER / 8; ++c)
+#pragma unroll
+                for (int k = 0; k < NV; ++k) r.v[c * NV + k] = __ldg(src + (size_t)(tid + c * NT) * NV + k);
+            return true;
+        };
+        nxt_fast = issue(s_begin, nxt);
+        for (int sl = s_begin; sl < s_end; ++sl) {
+            const RawItem<DT> cur = nxt;
+            const bool fast = nxt_fast;
+            nxt_fast = issue(sl + 1, nxt);
+            float z[PER];
+            if (fast) {
+#pragma unroll
+                for (int c = 0; c < PER / 8; ++c) {
+                    if (DT == SPEC_BF16) {
+                        const uint4 r = cur.v[c];
+                        z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
+                        z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
+                    } else {
+                        const uint4 r0 = cur.v[c * NV], r1 = cur.v[c * NV + NV - 1];
+                        z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
+                        z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
+                    }
+                }
+            } else {
+                // ragged or misaligned slice: whole chunks by 16-byte loads where they fit, else one logit at a time
+                const int n = min(SLICE, P.V - sl * SLICE);
+                const unsigned char *src = rowp + (size_t)sl * SLICE * ESZ;
+#pragma unroll
+                for (int c = 0; c < PER / 8; ++c) {
+                    const int t0 = (tid + c * NT) * 8;
+                    if (aligned && t0 + 8 <= n) {
+                        const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(tid + c * NT) * NV;
+                        if (DT == SPEC_BF16) {
+                            const uint4 r = __ldg(s4);
+                            z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
+                            z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
+                        } else {
+                            const uint4 r0 = __ldg(s4), r1 = __ldg(s4 + NV - 1);
+                            z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
+                            z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
+                    }
+                }
+            }
+            float zm = -CUDART_INF_F;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                bad |= (z[k] != z[k]) || (z[k] == CUDART_INF_F);
+                zm = fmaxf(zm, z[k]);
+            }
+            if (zm > -CUDART_INF_F) {
+                const float onew = fminf(fmaxf(ceilf(zm * s_hi), -1.0e9f), 1.0e9f);
+                if (!set) { of = onew; set = true; }
+                else if (onew > of) {
+                    // raise the reference: what was summed so far shrinks by an exact power of two
+                    const float dlt = of - onew;
+                    const float f = pow2i((int)fmaxf(dlt, -127.f));
+                    X_t = f * fmaf(dlt, S_t, X_t);
+                    S_t *= f;
+                    xm_t += dlt;
+                    of = onew;
+                }
+                xm_t = fmaxf(xm_t, fmaf(zm, s_lo, fmaf(zm, s_hi, -of)));
+            }
+            float sum[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int k = 0; k < PER; ++k) {
+                const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
+                const float e = ex2_approx(x);
+                sum[k & 3] += e;
+                sx[k & 3] = fmaf(e, x, sx[k & 3]);
+            }
+            S_t += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+            X_t += (sx[0] + sx[1]) + (sx[2] + sx[3]);
+        }
+        const int o_t = set ? (int)of : ROWPART_EMPTY;
+
+        // ---- warp, then CTA: merge (reference, sums) pairs by exact powers of two --------------------------------
+        const int O_w = __reduce_max_sync(0xffffffffu, o_t);
+        const int d = max(o_t - O_w, -100000);
+        const double f = (double)pow2i(max(d, -127));
+        const double Sw = warp_sum((double)S_t * f);
+        const double Xw = warp_sum(f * ((double)X_t + (double)d * (double)S_t));
+        double best = set ? (double)o_t + (double)xm_t : -1.0e300;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
+        bad = __any_sync(0xffffffffu, bad);
+        __syncthreads();             // the previous item's partials have been read
+        if (lane == 0) { sS[w] = Sw; sX[w] = Xw; sB[w] = best; sO[w] = O_w; sBad[w] = bad; }
+        __syncthreads();
+        if (tid == 0) {
+            int O = ROWPART_EMPTY, bd = 0;
+            double bst = -1.0e300;
+            for (int k = 0; k < NT / 32; ++k) { O = max(O, sO[k]); bd |= sBad[k]; bst = fmax(bst, sB[k]); }
+            double S = 0.0, X = 0.0;
+            for (int k = 0; k < NT / 32; ++k) {
+                const int dk = max(sO[k] - O, -100000);
+                const double fk = pow2d(dk);
+                S += sS[k] * fk;
+                X += fk * (sX[k] + (double)dk * sS[k]);
+            }
+            RowPart r;
+            r.S = S; r.X = X; r.O = O; r.xmax = O > ROWPART_EMPTY ? (float)(bst - (double)O) : 0.f;
+            r.cut = -CUDART_INF_F; r.bad = bd;
+            *out = r;
         }
     }
-    const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-    float s_hi = (float)s_d;
-    if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
-    float s_lo = (float)(s_d - (double)s_hi);
-    if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
+}
 
-    float zm = -CUDART_INF_F;
-    int bad = 0;
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        bad |= (z[k] != z[k]) || (z[k] == CUDART_INF_F);
-        zm = fmaxf(zm, z[k]);
-    }
-    const bool any = zm > -CUDART_INF_F;
-    const float of = any ? fminf(fmaxf(ceilf(zm * s_hi), -1.0e9f), 1.0e9f) : 0.f;
-    const int o_t = any ? (int)of : ROWPART_EMPTY;
-    float sum[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
-        const float e = ex2_approx(x);
-        sum[k & 3] += e;
-        sx[k & 3] = fmaf(e, x, sx[k & 3]);
-    }
-    const float S_t = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-    const float X_t = (sx[0] + sx[1]) + (sx[2] + sx[3]);
-    const float xm_t = fmaf(zm, s_lo, fmaf(zm, s_hi, -of));
+// Merge the slices of every row into one record (slice 0 of the merged array): one warp per row.
+struct MParams {
+    long long rows2;
+    int NSL;
+    const RowPart *part;     // [rows2][NSL]
+    RowPart *merged;         // [rows2]
+};
 
-    // ---- warp, then CTA: merge (reference, sums) pairs by exact powers of two ------------------------------------
-    const int O_w = __reduce_max_sync(0xffffffffu, o_t);
-    const int d = max(o_t - O_w, -100000);
-    const double f = (double)pow2i(max(d, -127));
-    const double Sw = warp_sum((double)S_t * f);
-    const double Xw = warp_sum(f * ((double)X_t + (double)d * (double)S_t));
-    double best = any ? (double)o_t + (double)xm_t : -1.0e300;
+__global__ void spec_row_merge_kernel(const MParams P)
+{
+    const long long r2 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r2 >= P.rows2) return;
+    const RowPart *p = P.part + r2 * P.NSL;
+    int O = ROWPART_EMPTY, bad = 0, unread = 0;
+    for (int j = lane; j < P.NSL; j += 32) { O = max(O, p[j].O); bad |= p[j].bad == 1; unread |= p[j].bad == -1; }
+    O = __reduce_max_sync(0xffffffffu, O);
+    bad = __any_sync(0xffffffffu, bad);
+    unread = __any_sync(0xffffffffu, unread);
+    double S = 0.0, X = 0.0, best = -1.0e300;
+    for (int j = lane; j < P.NSL; j += 32) {
+        if (p[j].O > ROWPART_EMPTY) {
+            const int d = max(p[j].O - O, -100000);
+            const double fk = pow2d(d);
+            S += p[j].S * fk;
+            X += fk * (p[j].X + (double)d * p[j].S);
+            best = fmax(best, (double)p[j].O + (double)p[j].xmax);
+        }
+    }
+    S = warp_sum(S);
+    X = warp_sum(X);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
-    bad = __any_sync(0xffffffffu, bad);
-    if (lane == 0) { sS[w] = Sw; sX[w] = Xw; sB[w] = best; sO[w] = O_w; sBad[w] = bad; }
-    __syncthreads();
-    if (tid == 0) {
-        int O = ROWPART_EMPTY, bd = 0;
-        double bst = -1.0e300;
-        for (int k = 0; k < NT / 32; ++k) { O = max(O, sO[k]); bd |= sBad[k]; bst = fmax(bst, sB[k]); }
-        double S = 0.0, X = 0.0;
-        for (int k = 0; k < NT / 32; ++k) {
-            const int dk = max(sO[k] - O, -100000);
-            const double fk = pow2d(dk);
-            S += sS[k] * fk;
-            X += fk * (sX[k] + (double)dk * sS[k]);
-        }
+    if (lane == 0) {
         RowPart r;
-        r.S = S; r.X = X; r.O = O; r.xmax = O > ROWPART_EMPTY ? (float)(bst - (double)O) : 0.f;
-        r.cut = -CUDART_INF_F; r.bad = bd;
-        *out = r;
+        r.S = S; r.X = X; r.O = O; r.xmax = O > ROWPART_EMPTY ? (float)(best - (double)O) : 0.f;
+        r.cut = -CUDART_INF_F;
+        r.bad = unread ? -1 : ((bad || !(S > 0.0) || !(S < CUDART_INF)) ? 1 : 0);
+        P.merged[r2] = r;
     }
 }
 
