@@ -75,7 +75,7 @@ inline int up(int x, int m) { return (x + m - 1) / m * m; }
 // two CTAs per SM, 128 registers each) while a slice fits in TMAX tiles of 1792 tokens, fifteen
 // consumer warps (one CTA per SM) above that.  SPECVERIFY_CLUSTER / SPECVERIFY_WARPS (environment)
 // force a cluster size / consumer warp count for tuning.
-bool make_vplan(int V, int dtype, VPlan *p)
+bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bool whole_sm = false)
 {
     const int esz = dtype == SPEC_BF16 ? 2 : 4;
     int force_c = 0, force_nw = 0;
@@ -85,14 +85,14 @@ bool make_vplan(int V, int dtype, VPlan *p)
         const int NW = pass == 0 ? 7 : 15;
         if (force_nw && force_nw != NW) continue;
         const int tile = NW * 32 * 8;
-        const int budget = NW == 7 ? SMEM_2CTA : SMEM_1CTA;
+        const int budget = (NW == 7 && !whole_sm) ? SMEM_2CTA : SMEM_1CTA;
         for (int C = 1; C <= CMAX; C <<= 1) {
             if (force_c && force_c != C) continue;
             const int slice = up((V + C - 1) / C, 8);
             const int tiles = (slice + tile - 1) / tile;
             if (tiles > TMAX) continue;
             if (pass == 0 && C > 8) continue;          // prefer one CTA per SM over a non-portable cluster
-            const int off_x = up((int)sizeof(Hdr), 128);
+            const int off_x = up(hdr_bytes, 128);
             const int off_es = off_x + up(2 * C * NW * 10 * 8, 128);
             const int es_bytes = (tiles > RT ? tiles - RT : 0) * tile * 8;
             const int off_ring = off_es + es_bytes;
@@ -356,8 +356,16 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         sp.part = NSL > 1 ? parts : part;
         const long long items = 2ll * in->B * in->N * NSL;
         const unsigned grid = (unsigned)(items < (1ll << 20) ? items : (1ll << 20));
-        if (in->logits_dtype == SPEC_BF16) stream::spec_row_partial_kernel<SPEC_BF16><<<grid, stream::NT, 0, st>>>(sp);
-        else stream::spec_row_partial_kernel<SPEC_F32><<<grid, stream::NT, 0, st>>>(sp);
+        int prc;
+        const bool feat = out->node_features != nullptr;
+#define SPECV_STREAM(DTV, FT)                                                                                     \
+    do {                                                                                                          \
+        if ((prc = prepare_kernel(stream::spec_row_partial_kernel<DTV, FT>, 1, stream::Ring<DTV>::BYTES))) return prc; \
+        stream::spec_row_partial_kernel<DTV, FT><<<grid, stream::NT, stream::Ring<DTV>::BYTES, st>>>(sp);         \
+    } while (0)
+        if (in->logits_dtype == SPEC_BF16) { if (feat) SPECV_STREAM(SPEC_BF16, true); else SPECV_STREAM(SPEC_BF16, false); }
+        else { if (feat) SPECV_STREAM(SPEC_F32, true); else SPECV_STREAM(SPEC_F32, false); }
+#undef SPECV_STREAM
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
         if (NSL > 1) {
             stream::MParams mp = {2ll * in->B * in->N, NSL, parts, part};
@@ -399,7 +407,17 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char *w = (unsigned char *)ws;
     const bool diagnostics = out->residual || out->node_thr || out->node_w_in || out->margin;
-    if (allow_walk && mode == MODE_SPECINFER && !diagnostics) return verify_walk(in, out, w, L, pl, trunc, st);
+    if (allow_walk && mode == MODE_SPECINFER && !diagnostics && in->N <= NWALK) {
+        // the walk keeps one cluster per sequence busy: when all of them fit on the chip with one CTA
+        // per SM, each CTA may use the whole SM's shared memory for its ring
+        VPlan wpl;
+        if (!make_vplan(in->V, in->logits_dtype, &wpl, (int)sizeof(WHdr), false)) return SPEC_ERR_UNSUPPORTED;
+        if ((long long)in->B * wpl.C <= sm_count()) {
+            VPlan big;
+            if (make_vplan(in->V, in->logits_dtype, &big, (int)sizeof(WHdr), true) && big.C == wpl.C && big.NW == wpl.NW) wpl = big;
+        }
+        return verify_walk(in, out, w, L, wpl, trunc, st);
+    }
     if (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
         cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess) {
         cudaGetLastError();

@@ -1,7 +1,7 @@
 // Streaming row statistics (no truncation): every logit row the verifiers may touch is read once from
 // HBM, straight into registers, and reduced to per-slice partial sums of the row's softmax normaliser.
 // No residency, no clusters: a CTA streams a row (or a part of it) in slices of 8192 logits, 32 per thread,
-// the 16-byte loads of the next slice in flight while the current one is exponentiated.
+// the asynchronous copies of the next slices in flight while the current one is exponentiated.
 //
 // A thread turns its logits into e = 2^(z s - o) (s = log2(e)/T, o = ceil of its own largest z s, an
 // integer, so partial sums combine by exact powers of two) and the CTA writes, for its slice,
@@ -39,23 +39,45 @@ struct SParams {
     RowPart *part;           // [B*N*2][NSL]
 };
 
-// raw logits of one thread for one slice: PER / 8 chunks of 8
-template <int DT>
-struct RawItem {
-    uint4 v[DT == SPEC_BF16 ? PER / 8 : PER / 4];
+// depth of the per-thread staging ring and its size
+template <int DT> struct Ring {
+    static constexpr int NV = DT == SPEC_BF16 ? 1 : 2;         // 16-byte units per chunk of 8 logits
+    static constexpr int UNITS = (PER / 8) * NV;               // 16-byte units per thread and slice
+    static constexpr int DEPTH = DT == SPEC_BF16 ? 5 : 3;
+    static constexpr int BYTES = DEPTH * UNITS * NT * 16;
 };
 
-// One CTA per (row, part of the row): the part's slices of 8192 logits are streamed one after the other,
-// the loads of the next slice issued before the arithmetic of the current one; each thread keeps a
-// running (reference, sum) pair, rescaled by an exact power of two when a later slice raises its
-// reference, and the CTA reduces once per part.
-template <int DT>
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// One CTA per (row, part of the row).  The part's slices of 8192 logits are streamed one after the
+// other; every thread stages its own 32 logits of the next DEPTH - 1 slices in shared memory with
+// asynchronous 16-byte copies (a thread reads back only what it copied itself, so the ring needs no
+// barrier) and keeps a running (reference, sum) pair, rescaled by an exact power of two when a later
+// slice raises its reference.  The CTA reduces once per part.
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));     // a NaN operand yields the other one
+    return d;
+}
+
+// FEAT: also accumulate X (needed only by the entropy features).  Without it a NaN or +inf logit is
+// found from the sum itself (such a logit makes its e, and so the thread's sum, non-finite), which
+// keeps comparisons out of the inner loop.
+template <int DT, bool FEAT>
 __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P)
 {
     constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
-    constexpr int NV = DT == SPEC_BF16 ? 1 : 2;           // 16-byte loads per chunk of 8 logits
+    constexpr int NV = Ring<DT>::NV, UNITS = Ring<DT>::UNITS, DEPTH = Ring<DT>::DEPTH;
     __shared__ double sS[NT / 32], sX[NT / 32], sB[NT / 32];
     __shared__ int sO[NT / 32], sBad[NT / 32];
+    uint4 *ring = reinterpret_cast<uint4 *>(dyn_smem);            // [DEPTH][UNITS][NT]
+    const uint32_t ring_s = (uint32_t)__cvta_generic_to_shared(ring);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const long long items = 2ll * P.B * P.N * P.NSL;
     const int slices_row = (P.V + SLICE - 1) / SLICE;
@@ -93,68 +115,91 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         bool set = false;
         int bad = 0;
 
-        RawItem<DT> nxt;
-        bool nxt_fast = false;
-        auto issue = [&](int sl, RawItem<DT> &r) -> bool {
-            if (sl >= s_end) return false;
-            const int n = min(SLICE, P.V - sl * SLICE);
-            if (!aligned || n < SLICE) return false;
-            const uint4 *src = reinterpret_cast<const uint4 *>(rowp + (size_t)sl * SLICE * ESZ);
+        // stage the thread's share of slice sl (16-byte units past the row's end are not copied; a unit
+        // that straddles it is zero-filled and masked by token index when it is used)
+        auto issue = [&](int sl) {
+            if (aligned && sl < s_end) {
+                const long long bytes_left = ((long long)P.V - (long long)sl * SLICE) * ESZ;
+                const unsigned char *src = rowp + (size_t)sl * SLICE * ESZ;
+                const uint32_t dst = ring_s + (uint32_t)(((sl - s_begin) % DEPTH) * UNITS * NT + tid) * 16u;
 #pragma unroll
-            for (int c = 0; c < PER / 8; ++c)
+                for (int c = 0; c < PER / 8; ++c)
 #pragma unroll
-                for (int k = 0; k < NV; ++k) r.v[c * NV + k] = __ldg(src + (size_t)(tid + c * NT) * NV + k);
-            return true;
+                    for (int k = 0; k < NV; ++k) {
+                        const long long off = ((long long)(tid + c * NT) * NV + k) * 16;
+                        const long long left = bytes_left - off;
+                        if (left > 0) cp_async16(dst + (uint32_t)((c * NV + k) * NT) * 16u, src + off, left < 16 ? (int)left : 16);
+                    }
+            }
+            cp_async_commit();
         };
-        nxt_fast = issue(s_begin, nxt);
+#pragma unroll
+        for (int k = 0; k < DEPTH - 1; ++k) issue(s_begin + k);
+
         for (int sl = s_begin; sl < s_end; ++sl) {
-            const RawItem<DT> cur = nxt;
-            const bool fast = nxt_fast;
-            nxt_fast = issue(sl + 1, nxt);
+            const int n = min(SLICE, P.V - sl * SLICE);
             float z[PER];
-            if (fast) {
+            float zm = -CUDART_INF_F;
+            if (aligned) {
+                cp_async_wait<DEPTH - 2>();
+                const uint4 *st = ring + (size_t)((sl - s_begin) % DEPTH) * UNITS * NT + tid;
+                uint4 raw[UNITS];
+#pragma unroll
+                for (int u = 0; u < UNITS; ++u) raw[u] = st[u * NT];
+                // the stage read in the previous iteration is free again
+                issue(sl + DEPTH - 1);
+                if (n < SLICE) {
+                    // ragged last slice: logits past the row's end count as -inf
+#pragma unroll
+                    for (int u = 0; u < UNITS; ++u) {
+                        const int t0 = DT == SPEC_BF16 ? (tid + u * NT) * 8 : (tid + (u / NV) * NT) * 8 + (u % NV) * 4;
+                        uint32_t *wd = reinterpret_cast<uint32_t *>(&raw[u]);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            if (DT == SPEC_BF16) {
+                                if (t0 + 2 * k >= n) wd[k] = (wd[k] & 0xFFFF0000u) | 0xFF80u;
+                                if (t0 + 2 * k + 1 >= n) wd[k] = (wd[k] & 0x0000FFFFu) | 0xFF800000u;
+                            } else if (t0 + k >= n) wd[k] = 0xFF800000u;
+                        }
+                    }
+                }
+                if (DT == SPEC_BF16) {
+                    // the slice maximum on packed pairs
+                    uint32_t m2 = 0xFF80FF80u;
+#pragma unroll
+                    for (int c = 0; c < PER / 8; ++c) {
+                        const uint4 r = raw[c];
+                        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(r.x, r.y), max_bf16x2(r.z, r.w)));
+                    }
+                    zm = fmaxf(bf16_lo(m2), bf16_hi(m2));
+                }
 #pragma unroll
                 for (int c = 0; c < PER / 8; ++c) {
                     if (DT == SPEC_BF16) {
-                        const uint4 r = cur.v[c];
+                        const uint4 r = raw[c];
                         z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
                         z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
                     } else {
-                        const uint4 r0 = cur.v[c * NV], r1 = cur.v[c * NV + NV - 1];
+                        const uint4 r0 = raw[c * NV], r1 = raw[c * NV + NV - 1];
                         z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
                         z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
                     }
                 }
             } else {
-                // ragged or misaligned slice: whole chunks by 16-byte loads where they fit, else one logit at a time
-                const int n = min(SLICE, P.V - sl * SLICE);
+                // misaligned row: one logit at a time
                 const unsigned char *src = rowp + (size_t)sl * SLICE * ESZ;
 #pragma unroll
                 for (int c = 0; c < PER / 8; ++c) {
                     const int t0 = (tid + c * NT) * 8;
-                    if (aligned && t0 + 8 <= n) {
-                        const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(tid + c * NT) * NV;
-                        if (DT == SPEC_BF16) {
-                            const uint4 r = __ldg(s4);
-                            z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
-                            z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
-                        } else {
-                            const uint4 r0 = __ldg(s4), r1 = __ldg(s4 + NV - 1);
-                            z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
-                            z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
-                        }
-                    } else {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
-                    }
+                    for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
                 }
             }
-            float zm = -CUDART_INF_F;
+            if (DT != SPEC_BF16 || !aligned) {
 #pragma unroll
-            for (int k = 0; k < PER; ++k) {
-                bad |= (z[k] != z[k]) || (z[k] == CUDART_INF_F);
-                zm = fmaxf(zm, z[k]);
+                for (int k = 0; k < PER; ++k) zm = fmaxf(zm, z[k]);
             }
+            bad |= zm == CUDART_INF_F;
             if (zm > -CUDART_INF_F) {
                 const float onew = fminf(fmaxf(ceilf(zm * s_hi), -1.0e9f), 1.0e9f);
                 if (!set) { of = onew; set = true; }
@@ -170,16 +215,25 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
                 xm_t = fmaxf(xm_t, fmaf(zm, s_lo, fmaf(zm, s_hi, -of)));
             }
             float sum[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
+            if (FEAT) {
 #pragma unroll
-            for (int k = 0; k < PER; ++k) {
-                const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
-                const float e = ex2_approx(x);
-                sum[k & 3] += e;
-                sx[k & 3] = fmaf(e, x, sx[k & 3]);
+                for (int k = 0; k < PER; ++k) {
+                    const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
+                    bad |= z[k] != z[k];
+                    const float e = ex2_approx(x);
+                    sum[k & 3] += e;
+                    sx[k & 3] = fmaf(e, x, sx[k & 3]);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < PER; ++k) sum[k & 3] += ex2_approx(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)));
             }
             S_t += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             X_t += (sx[0] + sx[1]) + (sx[2] + sx[3]);
         }
+        // a NaN logit leaves a NaN in the sum; +inf was seen in the maximum
+        bad |= !(fabsf(S_t) <= 3.0e38f);
+        cp_async_wait<0>();
         const int o_t = set ? (int)of : ROWPART_EMPTY;
 
         // ---- warp, then CTA: merge (reference, sums) pairs by exact powers of two --------------------------------

@@ -9,6 +9,11 @@
 // where Algorithm 4 needs a residual: at a node whose first child was rejected, and at the stop node
 // for the bonus draw.  That is one or two resident nodes per sequence instead of every node of the tree.
 //
+// Before the walk the consumer threads of every CTA bring the sequence's scalars into shared memory in
+// two rounds of independent loads: topology, tokens, uniforms and the row records; then, for every
+// non-root node, the two logits at its token in its parent's rows, turned into final probabilities.
+// After that a step down the tree is a few shared-memory reads.
+//
 // Every consumer warp of the cluster runs the same walk on the same numbers (the exchanges deliver
 // bit-identical totals to all of them), so control flow agrees across the cluster without barriers.
 // The thread that finds the bonus token writes all outputs of the sequence.
@@ -17,6 +22,8 @@
 #include "verify.cuh"
 
 namespace specv {
+
+constexpr int NWALK = 128;        // nodes per sequence the walk keeps in shared memory
 
 struct WParams {
     int B, N, V, C, NSL;
@@ -37,51 +44,22 @@ struct __align__(16) WHdr {
     WarpArea wa[NWMAX];
     int req_a, req_b, req_hq;
     int poison;
+    // the sequence's scalars (written by the prologue of every sequence)
+    int t_parent[NWALK], t_token[NWALK], t_fc[NWALK], t_kc[NWALK];
+    float t_u[NWALK], t_ub[NWALK];
+    double t_Z[2 * NWALK];        // normaliser of row (node, target / draft), in units of 2^O
+    int t_O[2 * NWALK];
+    float t_cut[2 * NWALK];
+    double t_cp[NWALK], t_cq[NWALK];   // probability of the node's token under its parent's p and q
+    int t_status;
 };
 
-// merged statistics of one row: reference, normaliser, cut, entropy sum, largest exponent, validity
+// statistics of one row: normaliser, reference, cut
 struct RowSum {
-    double Z, X;
+    double Z;
     int O;
-    float cut, xmax;
-    int bad;        // 1: NaN / +inf / no finite logit
+    float cut;
 };
-
-// every lane gets the same answer; lanes share the slices of the row
-__device__ __forceinline__ RowSum merge_row(const RowPart *part, long long row2, int NSL, int lane)
-{
-    int O = ROWPART_EMPTY, bad = 0;
-    float cutv = -CUDART_INF_F;
-    for (int j = lane; j < NSL; j += 32) {
-        const RowPart *p = part + row2 * NSL + j;
-        O = max(O, __ldcg(&p->O));
-        bad |= __ldcg(&p->bad) == 1;
-        if (j == 0) cutv = __ldcg(&p->cut);
-    }
-    O = __reduce_max_sync(0xffffffffu, O);
-    double S = 0.0, X = 0.0, best = -1.0e300;
-    for (int j = lane; j < NSL; j += 32) {
-        const RowPart *p = part + row2 * NSL + j;
-        const int o = __ldcg(&p->O);
-        if (o > ROWPART_EMPTY) {
-            const int d = max(o - O, -100000);
-            const double f = pow2d(d), s = __ldcg(&p->S);
-            S += s * f;
-            X += f * (__ldcg(&p->X) + (double)d * s);
-            best = fmax(best, (double)o + (double)__ldcg(&p->xmax));
-        }
-    }
-    RowSum r;
-    r.Z = warp_sum(S);
-    r.X = warp_sum(X);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
-    r.O = O;
-    r.cut = __shfl_sync(0xffffffffu, cutv, 0);
-    r.xmax = O > ROWPART_EMPTY ? (float)(best - (double)O) : 0.f;
-    r.bad = __any_sync(0xffffffffu, bad) || !(r.Z > 0.0) || !(r.Z < CUDART_INF);
-    return r;
-}
 
 template <int DT, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kernel(const WParams P)
@@ -198,32 +176,62 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
             float s_lo = (float)(s_d - (double)s_hi);
             if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
 
-            // ---- the whole tree is checked first: topology, tokens, rows that are not finite ------------------
-            int status = 0;
-            for (int i = lane; i < P.N; i += 32) {
-                const int pa = __ldg(parent + i);
-                if (i == 0 ? (pa != -1) : (pa < 0 || pa >= i)) status = max(status, SPEC_DEV_TOPOLOGY);
-                if (i > 0) {
-                    const int x = __ldg(token + i);
-                    if (x < 0 || x >= P.V) status = max(status, SPEC_DEV_TOKEN);
-                }
-            }
+            // ---- round 1: topology, tokens, uniforms, row records; the whole tree is checked ----------------------
+            bar_sync(1, NCONS);                      // the previous sequence's scalars are no longer read
+            if (tid == 0) S.t_status = 0;
+            bar_sync(1, NCONS);
             {
-                // a row is not finite if a slice saw NaN / +inf, or if no slice has a finite logit
-                const long long rows2 = 2ll * P.N;
-                for (long long r2 = lane; r2 < rows2; r2 += 32) {
-                    const RowPart *p = P.part + ((long long)b * rows2 + r2) * P.NSL;
-                    int any_finite = 0, bad = 0, unread = 0;
-                    for (int j = 0; j < P.NSL; ++j) {
-                        const int bd = __ldcg(&p[j].bad);
-                        unread |= bd == -1;
-                        bad |= bd == 1;
-                        any_finite |= __ldcg(&p[j].O) > ROWPART_EMPTY && __ldcg(&p[j].S) > 0.0;
+                int st1 = 0;
+                for (int i = tid; i < P.N; i += NCONS) {
+                    const int pa = __ldg(parent + i);
+                    if (i == 0 ? (pa != -1) : (pa < 0 || pa >= i)) st1 = max(st1, SPEC_DEV_TOPOLOGY);
+                    int x = 0;
+                    if (i > 0) {
+                        x = __ldg(token + i);
+                        if (x < 0 || x >= P.V) st1 = max(st1, SPEC_DEV_TOKEN);
                     }
-                    if (!unread && (bad || !any_finite)) status = max(status, SPEC_DEV_NONFINITE);
+                    S.t_parent[i] = pa; S.t_token[i] = x; S.t_fc[i] = P.N; S.t_kc[i] = 0;
+                    S.t_u[i] = __ldg(P.u_accept + (long long)b * P.N + i);
+                    S.t_ub[i] = __ldg(P.u_bonus + (long long)b * P.N + i);
                 }
+                for (int r2 = tid; r2 < 2 * P.N; r2 += NCONS) {
+                    const RowPart *p = P.part + ((long long)b * 2 * P.N + r2);
+                    const double Zr = __ldcg(&p->S);
+                    const int Or = __ldcg(&p->O), bd = __ldcg(&p->bad);
+                    // a row is not finite if it holds NaN / +inf, or no finite logit at all
+                    if (bd != -1 && (bd == 1 || !(Or > ROWPART_EMPTY) || !(Zr > 0.0) || !(Zr < CUDART_INF)))
+                        st1 = max(st1, SPEC_DEV_NONFINITE);
+                    S.t_Z[r2] = Zr; S.t_O[r2] = Or; S.t_cut[r2] = __ldcg(&p->cut);
+                }
+                if (st1) atomicMax(&S.t_status, st1);
             }
-            status = __reduce_max_sync(0xffffffffu, status);
+            bar_sync(1, NCONS);
+            // ---- round 2: children, and the probability of every node's token under its parent's rows -------------
+            if (S.t_status == 0) {
+                int st2 = 0;
+                for (int c = 1 + tid; c < P.N; c += NCONS) {
+                    const int a = S.t_parent[c], xt = S.t_token[c];
+                    atomicMin(&S.t_fc[a], c);
+                    if (atomicAdd(&S.t_kc[a], 1) >= KMAX) st2 = SPEC_DEV_TOPOLOGY;
+                    const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
+                    const float zp_x = load_logit(P.zp, DT, rowb + xt), zq_x = load_logit(P.zq, DT, rowb + xt);
+                    double pr[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const float z = h ? zq_x : zp_x;
+                        const double xd = (double)z * s_d - (double)S.t_O[2 * a + h];
+                        pr[h] = 0.0;
+                        if (z >= S.t_cut[2 * a + h] && xd > -1000.0) {
+                            const double nd = rint(xd);
+                            pr[h] = exp2_frac(xd - nd) * pow2d((int)nd) * __drcp_rn(S.t_Z[2 * a + h]);
+                        }
+                    }
+                    S.t_cp[c] = pr[0]; S.t_cq[c] = pr[1];
+                }
+                if (st2) atomicMax(&S.t_status, st2);
+            }
+            bar_sync(1, NCONS);
+            int status = S.t_status;
             int cur = 0, len = 0;
             int bonus = -1;
             bool writer = false;          // this lane writes the sequence's outputs
@@ -232,48 +240,14 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
 
             while (!done) {
                 const int a = cur;
-                // ---- children of a ------------------------------------------------------------------------------
-                int kc = 0;
-                for (int c0 = a + 1; c0 < P.N; c0 += 32) {
-                    const int c = c0 + lane;
-                    const bool is = c < P.N && __ldg(parent + c) == a;
-                    const unsigned bal = __ballot_sync(0xffffffffu, is);
-                    if (is) {
-                        const int pos = kc + __popc(bal & ((1u << lane) - 1u));
-                        if (pos < KMAX) {
-                            W.child[pos] = c;
-                            W.cpn[pos] = __ldg(token + c);
-                            W.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
-                        }
-                    }
-                    kc += __popc(bal);
-                }
-                if (kc > KMAX) { status = SPEC_DEV_TOPOLOGY; done = true; if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; } break; }
-                const bool hq = kc > 0;
-                const RowSum rp = merge_row(P.part, ((long long)b * P.N + a) * 2, P.NSL, lane);
-                RowSum rq = rp;
-                if (hq) rq = merge_row(P.part, ((long long)b * P.N + a) * 2 + 1, P.NSL, lane);
+                const int c_first = S.t_fc[a];
+                const bool hq = c_first < P.N;
+                const int kc = S.t_kc[a];
+                RowSum rp, rq;
+                rp.Z = S.t_Z[2 * a]; rp.O = S.t_O[2 * a]; rp.cut = S.t_cut[2 * a];
+                rq = rp;
+                if (hq) { rq.Z = S.t_Z[2 * a + 1]; rq.O = S.t_O[2 * a + 1]; rq.cut = S.t_cut[2 * a + 1]; }
                 const double invZp = __drcp_rn(rp.Z), invZq = hq ? __drcp_rn(rq.Z) : 0.0;
-                // target / draft probability of every child's token (lanes j and 16 + j)
-                __syncwarp();
-                {
-                    const int j = lane & 15;
-                    const bool mine = j < kc;
-                    const int xt = mine ? W.cpn[j] : 0;
-                    __syncwarp();
-                    if (mine) {
-                        const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
-                        const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + xt);
-                        const double xd = (double)z * s_d - (double)(lane < 16 ? rp.O : rq.O);
-                        double pr = 0.0;
-                        if (z >= (lane < 16 ? rp.cut : rq.cut) && xd > -1000.0) {
-                            const double nd = rint(xd);
-                            pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
-                        }
-                        if (lane < 16) W.cpm[j] = pr; else W.cqm[j] = pr;
-                    }
-                    __syncwarp();
-                }
                 // ---- first child: needs no residual -------------------------------------------------------------------
                 bool resident = false;
                 double st_c = 0.0, st_E = 1.0, g_commit = 0.0;
@@ -281,14 +255,30 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 int acc = -1;
                 int j0 = 0;
                 if (hq) {
-                    const double Pp = W.cpm[0], Pq = W.cqm[0];
+                    const double Pp = S.t_cp[c_first], Pq = S.t_cq[c_first];
                     const bool zero = !(Pp > 0.0), one = !zero && !(Pq > 0.0);
-                    if (!zero && (one || (double)W.cu[0] * Pq < Pp)) acc = W.child[0];
+                    if (!zero && (one || (double)S.t_u[c_first] * Pq < Pp)) acc = c_first;
                     j0 = 1;
                 }
                 if (acc < 0) {
                     // ---- the node comes on chip: e = 2^(z s - O) of both rows ----------------------------------------
                     resident = true;
+                    // the warp's list of the node's children, in index order
+                    if (kc > 1) {
+                        __syncwarp();
+                        int seen = 0;
+                        for (int c0 = a + 1; c0 < P.N && seen < kc; c0 += 32) {
+                            const int c = c0 + lane;
+                            const bool is = c < P.N && S.t_parent[c] == a;
+                            const unsigned bal = __ballot_sync(0xffffffffu, is);
+                            if (is) {
+                                const int pos = seen + __popc(bal & ((1u << lane) - 1u));
+                                W.child[pos] = c; W.cpm[pos] = S.t_cp[c]; W.cqm[pos] = S.t_cq[c]; W.cu[pos] = S.t_u[c];
+                            }
+                            seen += __popc(bal);
+                        }
+                        __syncwarp();
+                    }
                     if (warp == 0 && lane == 0) {
                         if (posted) { if (!mbar_wait(&S.ack, aphase)) S.poison = 1; aphase ^= 1u; }
                         S.req_a = a; S.req_b = b; S.req_hq = hq ? 1 : 0;
@@ -410,7 +400,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 // ---- stop here: the bonus token from the committed residual ---------------------------------------------
                 done = true;
                 const double E_tot = warp_sum(lane < C ? E_r : 0.0);
-                const double target = (double)__ldg(P.u_bonus + (long long)b * P.N + a) * E_tot;
+                const double target = (double)S.t_ub[a] * E_tot;
                 double tau;
                 const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
                 if (owner < 0) {
@@ -503,7 +493,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 if (accn >= 0) {
                     ot[ln] = bn;
                     int i = ln;
-                    for (int x = accn; x != 0 && i > 0; x = __ldg(parent + x)) ot[--i] = __ldg(token + x);
+                    for (int x = accn; x != 0 && i > 0; x = S.t_parent[x]) ot[--i] = S.t_token[x];
                 }
             }
         }
