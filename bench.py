@@ -29,7 +29,10 @@ METRIC = "verified tree-nodes/sec"
 UNIT = "nodes/s"
 L2_BYTES = 132_644_864
 ROTATE_BYTES = 4 * L2_BYTES          # bytes touched before an input copy is read again
-KERNELS_PER_CALL = 1                 # the fused verify kernel (the two memset nodes before it are not counted)
+# kernels of one call; the roofline figure is taken over the whole call (all of its kernels), so it
+# understates the fraction the streaming kernel reaches on its own
+KERNELS = {"specinfer": "spec_row_partial_kernel + spec_walk_kernel (whole specinfer call)",
+           "traversal": "spec_verify_kernel (whole traversal call)"}
 
 
 def parse_args():
@@ -42,6 +45,7 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU work spent on the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="enqueue every call from the host instead of replaying CUDA graphs")
     return ap.parse_args()
 
 
@@ -192,18 +196,66 @@ def run_ours(args):
                                            b.u_bonus, w.temperature, w.top_k, w.top_p, outputs=outs)
                     for b in batches] for a in w.algorithms}
     counter = [0]
+    for a in w.algorithms:               # first calls set kernel attributes: they must not fall inside a capture
+        for p in prepared[a]:
+            p.launch(stream)
+    torch.cuda.synchronize()
+    launches_per_step = None
+    if args.no_graph:
+        def call(algo):
+            p = prepared[algo][counter[0] % len(batches)]
+            counter[0] += 1
+            p.launch(stream)
 
-    def call(algo):
-        p = prepared[algo][counter[0] % len(batches)]
-        counter[0] += 1
-        p.launch(stream)
+        def step():
+            for algo in w.algorithms:
+                call(algo)
+    else:
+        # the library neither allocates nor synchronises, so a call can be captured: one graph per input
+        # copy for the whole step, one per (algorithm, copy) for the per-algorithm figures
+        side = torch.cuda.Stream()
 
-    def step():
-        for algo in w.algorithms:
-            call(algo)
+        def capture(algos, copies_):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for i in copies_:
+                        for a in algos:
+                            prepared[a][i].launch(side)
+            return g
 
-    for _ in range(max(3, args.warmup)):
-        step()
+        every = list(range(len(batches)))
+        before = binding.kernel_launches()
+        step_graphs = [capture(w.algorithms, [i]) for i in every]
+        launches_per_step = (binding.kernel_launches() - before) // len(batches)
+        # a round over all input copies as one graph: consecutive steps then follow each other on the
+        # device without a host launch in between
+        round_graph = capture(w.algorithms, every)
+        algo_round = {a: capture([a], every) for a in w.algorithms}
+        algo_single = {a: [capture([a], [i]) for i in every] for a in w.algorithms}
+
+        def run_steps(n):
+            for _ in range(n // len(batches)):
+                round_graph.replay()
+            for i in range(n % len(batches)):
+                step_graphs[i].replay()
+
+        def run_calls(algo, n):
+            for _ in range(n // len(batches)):
+                algo_round[algo].replay()
+            for i in range(n % len(batches)):
+                algo_single[algo][i].replay()
+
+    if args.no_graph:
+        def run_steps(n):
+            for _ in range(n):
+                step()
+
+        def run_calls(algo, n):
+            for _ in range(n):
+                call(algo)
+
+    run_steps(max(3, args.warmup))
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -212,23 +264,23 @@ def run_ours(args):
     shard.barrier(world)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = binding.kernel_launches()
     e0.record(stream)
-    for _ in range(args.steps):
-        step()
+    run_steps(args.steps)
     e1.record(stream)
     torch.cuda.synchronize()
+    # counted by the library at every launch site (for graphs: at capture, times the replays)
+    gpu_launches = (binding.kernel_launches() - launches0) if launches_per_step is None else launches_per_step * args.steps
     shard.barrier(world)
     ms_total = shard.max_over_ranks(e0.elapsed_time(e1), world, dev)
     # per-algorithm call duration (the node kernel dominates a call), same rotation of cold inputs
     per_algo = {}
     for algo in w.algorithms:
-        for _ in range(3):
-            call(algo)
+        run_calls(algo, max(3, len(batches)))
         torch.cuda.synchronize()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record(stream)
-        for _ in range(args.steps):
-            call(algo)
+        run_calls(algo, args.steps)
         a1.record(stream)
         torch.cuda.synchronize()
         ms = a0.elapsed_time(a1) / args.steps
@@ -286,16 +338,19 @@ def run_ours(args):
         "config": {"workload": w.name, "B_per_gpu": w.B, "N": w.N, "V": w.V, "logits": w.dtype,
                    "tree": f"delayed K={w.K} L1={w.L1} L2={w.L2}", "temperature": w.temperature, "top_k": w.top_k,
                    "top_p": w.top_p, "step": "+".join(w.algorithms) + " on one batch",
+                   "launch": "host enqueue per call" if args.no_graph else
+                             f"CUDA graph replay: one graph holds a round of {len(batches)} steps (one per input copy), "
+                             "single-step graphs for the remainder",
                    "node_verifications_per_step": nodes_per_step, "logit_bytes_per_call": bytes_per_call,
                    "l2": f"{copies} input copies rotated ({copies * bytes_per_call / 1e6:.0f} MB touched between "
                          f"reuses, L2 is {L2_BYTES / 1e6:.0f} MB)" if copies > 1 else "inputs larger than L2"},
         "hbm_gbs": world * bytes_per_call * len(w.algorithms) / ms_per_step / 1e6,
         "per_algorithm": per_algo,
-        "roofline": {"bound": "hbm", "kernel": f"spec_verify_kernel ({dom} call)", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": KERNELS[dom], "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": None,
                      "algorithmic_bytes_per_launch": bytes_per_call},
-        "clocks": clocks, "gpu_launches": KERNELS_PER_CALL * len(w.algorithms) * args.steps,
+        "clocks": clocks, "gpu_launches": gpu_launches,
         "status_ok": status_ok,
     }
     if e2e is not None:

@@ -197,6 +197,10 @@ int32_t spec_verify_host(const SpecIn *in, const SpecOut *out, int32_t algorithm
 int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, int32_t *slice_len,
                         int32_t *smem_bytes, int32_t *threads);
 
+/* Number of kernels this library has enqueued in the calling process so far (host-only counter, for
+ * benchmarks that report how many launches a timed region made).  Never fails. */
+int64_t spec_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

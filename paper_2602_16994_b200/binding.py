@@ -26,7 +26,7 @@ ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR
           -4: "SPEC_ERR_PARAM", -5: "SPEC_ERR_WORKSPACE", -6: "SPEC_ERR_UNSUPPORTED", -7: "SPEC_ERR_CUDA"}
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
            "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
-           "spec_verify_specinfer_static")
+           "spec_verify_specinfer_static", "spec_kernel_launches")
 
 
 class SpecIn(C.Structure):
@@ -77,6 +77,8 @@ def load_library(path: str = LIB_PATH):
                                       C.c_void_p, C.c_int64, C.c_void_p]
     lib.spec_query_plan.restype = C.c_int32
     lib.spec_query_plan.argtypes = [C.c_int32, C.c_int32] + [C.POINTER(C.c_int32)] * 4
+    lib.spec_kernel_launches.restype = C.c_int64
+    lib.spec_kernel_launches.argtypes = []
     lib.spec_host_staging_bytes.restype = C.c_int32
     lib.spec_host_staging_bytes.argtypes = [C.POINTER(SpecIn), C.POINTER(C.c_int64)]
     lib.spec_verify_host.restype = C.c_int32
@@ -103,6 +105,11 @@ def _ptr(t):
 def _stream_ptr(stream):
     s = stream if stream is not None else torch.cuda.current_stream()
     return C.c_void_p(s.cuda_stream)
+
+
+def kernel_launches() -> int:
+    """Kernels the library has enqueued in this process so far."""
+    return int(load_library().spec_kernel_launches())
 
 
 def query_plan(V: int, dtype: int = SPEC_BF16) -> dict:

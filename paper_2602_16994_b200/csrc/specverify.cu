@@ -8,6 +8,7 @@
 #include <stdint.h>
 #include <stdlib.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -169,6 +170,9 @@ WsLayout ws_layout(const SpecIn *in, int slices = 32)   // slices = 0: merged ro
     return L;
 }
 
+// kernels enqueued by the library in this process (benchmarks report it)
+std::atomic<long long> g_kernel_launches{0};
+
 template <typename K>
 int launch_clustered(K kernel, int ctas, int C, int threads, int smem, cudaStream_t st, void *params_ptr)
 {
@@ -187,6 +191,7 @@ int launch_clustered(K kernel, int ctas, int C, int threads, int smem, cudaStrea
     void *args[1] = {params_ptr};
     cudaError_t e = cudaLaunchKernelExC(&cfg, (const void *)kernel, args);
     if (e != cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
     return SPEC_OK;
 }
 
@@ -362,6 +367,7 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
     do {                                                                                                          \
         if ((prc = prepare_kernel(stream::spec_row_partial_kernel<DTV, FT>, 1, stream::Ring<DTV>::BYTES))) return prc; \
         stream::spec_row_partial_kernel<DTV, FT><<<grid, stream::NT, stream::Ring<DTV>::BYTES, st>>>(sp);         \
+        g_kernel_launches.fetch_add(1, std::memory_order_relaxed);                                               \
     } while (0)
         if (in->logits_dtype == SPEC_BF16) { if (feat) SPECV_STREAM(SPEC_BF16, true); else SPECV_STREAM(SPEC_BF16, false); }
         else { if (feat) SPECV_STREAM(SPEC_F32, true); else SPECV_STREAM(SPEC_F32, false); }
@@ -370,6 +376,7 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         if (NSL > 1) {
             stream::MParams mp = {2ll * in->B * in->N, NSL, parts, part};
             stream::spec_row_merge_kernel<<<(unsigned)((mp.rows2 * 32 + 255) / 256), 256, 0, st>>>(mp);
+            g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
             if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
         }
         NSL = 1;
@@ -378,6 +385,7 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         stream::FParams fp = {(long long)in->B * in->N, NSL, part, out->node_features};
         const unsigned grid = (unsigned)(((long long)in->B * in->N * 32 + 255) / 256);
         stream::spec_features_kernel<<<grid, 256, 0, st>>>(fp);
+        g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     }
     WParams wp = {};
@@ -463,6 +471,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         int gx = (in->V + 255) / 256;
         if (gx > 296) gx = 296;
         spec_residual_kernel<<<dim3(gx, in->B), 256, 0, st>>>(rp);
+        g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     }
     return SPEC_OK;
@@ -554,6 +563,8 @@ int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, 
     if (threads) *threads = (pl.NW + 1) * 32;
     return SPEC_OK;
 }
+
+int64_t spec_kernel_launches(void) { return (int64_t)g_kernel_launches.load(std::memory_order_relaxed); }
 
 int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream)
 {

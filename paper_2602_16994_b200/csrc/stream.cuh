@@ -115,96 +115,13 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         bool set = false;
         int bad = 0;
 
-        // stage the thread's share of slice sl (16-byte units past the row's end are not copied; a unit
-        // that straddles it is zero-filled and masked by token index when it is used)
-        auto issue = [&](int sl) {
-            if (aligned && sl < s_end) {
-                const long long bytes_left = ((long long)P.V - (long long)sl * SLICE) * ESZ;
-                const unsigned char *src = rowp + (size_t)sl * SLICE * ESZ;
-                const uint32_t dst = ring_s + (uint32_t)(((sl - s_begin) % DEPTH) * UNITS * NT + tid) * 16u;
-#pragma unroll
-                for (int c = 0; c < PER / 8; ++c)
-#pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        const long long off = ((long long)(tid + c * NT) * NV + k) * 16;
-                        const long long left = bytes_left - off;
-                        if (left > 0) cp_async16(dst + (uint32_t)((c * NV + k) * NT) * 16u, src + off, left < 16 ? (int)left : 16);
-                    }
-            }
-            cp_async_commit();
-        };
-#pragma unroll
-        for (int k = 0; k < DEPTH - 1; ++k) issue(s_begin + k);
-
-        for (int sl = s_begin; sl < s_end; ++sl) {
-            const int n = min(SLICE, P.V - sl * SLICE);
-            float z[PER];
-            float zm = -CUDART_INF_F;
-            if (aligned) {
-                cp_async_wait<DEPTH - 2>();
-                const uint4 *st = ring + (size_t)((sl - s_begin) % DEPTH) * UNITS * NT + tid;
-                uint4 raw[UNITS];
-#pragma unroll
-                for (int u = 0; u < UNITS; ++u) raw[u] = st[u * NT];
-                // the stage read in the previous iteration is free again
-                issue(sl + DEPTH - 1);
-                if (n < SLICE) {
-                    // ragged last slice: logits past the row's end count as -inf
-#pragma unroll
-                    for (int u = 0; u < UNITS; ++u) {
-                        const int t0 = DT == SPEC_BF16 ? (tid + u * NT) * 8 : (tid + (u / NV) * NT) * 8 + (u % NV) * 4;
-                        uint32_t *wd = reinterpret_cast<uint32_t *>(&raw[u]);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            if (DT == SPEC_BF16) {
-                                if (t0 + 2 * k >= n) wd[k] = (wd[k] & 0xFFFF0000u) | 0xFF80u;
-                                if (t0 + 2 * k + 1 >= n) wd[k] = (wd[k] & 0x0000FFFFu) | 0xFF800000u;
-                            } else if (t0 + k >= n) wd[k] = 0xFF800000u;
-                        }
-                    }
-                }
-                if (DT == SPEC_BF16) {
-                    // the slice maximum on packed pairs
-                    uint32_t m2 = 0xFF80FF80u;
-#pragma unroll
-                    for (int c = 0; c < PER / 8; ++c) {
-                        const uint4 r = raw[c];
-                        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(r.x, r.y), max_bf16x2(r.z, r.w)));
-                    }
-                    zm = fmaxf(bf16_lo(m2), bf16_hi(m2));
-                }
-#pragma unroll
-                for (int c = 0; c < PER / 8; ++c) {
-                    if (DT == SPEC_BF16) {
-                        const uint4 r = raw[c];
-                        z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
-                        z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
-                    } else {
-                        const uint4 r0 = raw[c * NV], r1 = raw[c * NV + NV - 1];
-                        z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
-                        z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
-                    }
-                }
-            } else {
-                // misaligned row: one logit at a time
-                const unsigned char *src = rowp + (size_t)sl * SLICE * ESZ;
-#pragma unroll
-                for (int c = 0; c < PER / 8; ++c) {
-                    const int t0 = (tid + c * NT) * 8;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
-                }
-            }
-            if (DT != SPEC_BF16 || !aligned) {
-#pragma unroll
-                for (int k = 0; k < PER; ++k) zm = fmaxf(zm, z[k]);
-            }
+        // a slice's maximum moves the thread's reference up by an exact power of two
+        auto new_reference = [&](float zm) {
             bad |= zm == CUDART_INF_F;
             if (zm > -CUDART_INF_F) {
                 const float onew = fminf(fmaxf(ceilf(zm * s_hi), -1.0e9f), 1.0e9f);
                 if (!set) { of = onew; set = true; }
                 else if (onew > of) {
-                    // raise the reference: what was summed so far shrinks by an exact power of two
                     const float dlt = of - onew;
                     const float f = pow2i((int)fmaxf(dlt, -127.f));
                     X_t = f * fmaf(dlt, S_t, X_t);
@@ -212,28 +129,139 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
                     xm_t += dlt;
                     of = onew;
                 }
-                xm_t = fmaxf(xm_t, fmaf(zm, s_lo, fmaf(zm, s_hi, -of)));
+                if (FEAT) xm_t = fmaxf(xm_t, fmaf(zm, s_lo, fmaf(zm, s_hi, -of)));
             }
-            float sum[4] = {0.f, 0.f, 0.f, 0.f}, sx[4] = {0.f, 0.f, 0.f, 0.f};
+        };
+        // 8 logits into the sums
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f, b0 = 0.f, b1 = 0.f;
+        auto add8 = [&](const float (&z)[8]) {
             if (FEAT) {
 #pragma unroll
-                for (int k = 0; k < PER; ++k) {
+                for (int k = 0; k < 8; ++k) {
                     const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
                     bad |= z[k] != z[k];
                     const float e = ex2_approx(x);
-                    sum[k & 3] += e;
-                    sx[k & 3] = fmaf(e, x, sx[k & 3]);
+                    if (k & 1) { a1 += e; b1 = fmaf(e, x, b1); } else { a0 += e; b0 = fmaf(e, x, b0); }
                 }
             } else {
-#pragma unroll
-                for (int k = 0; k < PER; ++k) sum[k & 3] += ex2_approx(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)));
+                a0 += ex2_approx(fmaf(z[0], s_lo, fmaf(z[0], s_hi, -of)));
+                a1 += ex2_approx(fmaf(z[1], s_lo, fmaf(z[1], s_hi, -of)));
+                a2 += ex2_approx(fmaf(z[2], s_lo, fmaf(z[2], s_hi, -of)));
+                a3 += ex2_approx(fmaf(z[3], s_lo, fmaf(z[3], s_hi, -of)));
+                a0 += ex2_approx(fmaf(z[4], s_lo, fmaf(z[4], s_hi, -of)));
+                a1 += ex2_approx(fmaf(z[5], s_lo, fmaf(z[5], s_hi, -of)));
+                a2 += ex2_approx(fmaf(z[6], s_lo, fmaf(z[6], s_hi, -of)));
+                a3 += ex2_approx(fmaf(z[7], s_lo, fmaf(z[7], s_hi, -of)));
             }
-            S_t += (sum[0] + sum[1]) + (sum[2] + sum[3]);
-            X_t += (sx[0] + sx[1]) + (sx[2] + sx[3]);
+        };
+        auto flush = [&]() {
+            S_t += (a0 + a1) + (a2 + a3);
+            X_t += b0 + b1;
+            a0 = a1 = a2 = a3 = b0 = b1 = 0.f;
+        };
+
+        // ---- whole slices of an aligned row go through the ring ------------------------------------------------
+        const int tok_end = min(P.V, s_end * SLICE);                       // first token past this part
+        const int nfull = aligned ? max(0, (tok_end - s_begin * SLICE) / SLICE) : 0;
+        {
+            const unsigned char *src = rowp + (size_t)s_begin * SLICE * ESZ + (size_t)tid * 16 * NV;
+            const uint32_t dst0 = ring_s + (uint32_t)tid * 16u;
+            int isl = 0, ist = 0, cst = 0;
+            auto issue = [&]() {
+                if (isl < nfull) {
+#pragma unroll
+                    for (int c = 0; c < PER / 8; ++c)
+#pragma unroll
+                        for (int k = 0; k < NV; ++k)
+                            cp_async16(dst0 + (uint32_t)((ist * UNITS + c * NV + k) * NT) * 16u, src + (size_t)c * NT * 16 * NV + k * 16, 16);
+                    src += (size_t)SLICE * ESZ;
+                    ++isl;
+                    ist = ist + 1 == DEPTH ? 0 : ist + 1;
+                }
+                cp_async_commit();
+            };
+#pragma unroll
+            for (int k = 0; k < DEPTH - 1; ++k) issue();
+            for (int sl = 0; sl < nfull; ++sl) {
+                cp_async_wait<DEPTH - 2>();
+                const uint4 *st = ring + (size_t)cst * UNITS * NT + tid;
+                uint4 raw[UNITS];
+#pragma unroll
+                for (int u = 0; u < UNITS; ++u) raw[u] = st[u * NT];
+                cst = cst + 1 == DEPTH ? 0 : cst + 1;
+                issue();                                  // the stage read in the previous iteration is free again
+                float zm;
+                if (DT == SPEC_BF16) {
+                    uint32_t m2 = 0xFF80FF80u;            // the slice maximum on packed pairs
+#pragma unroll
+                    for (int u = 0; u < UNITS; ++u)
+                        m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(raw[u].x, raw[u].y), max_bf16x2(raw[u].z, raw[u].w)));
+                    zm = fmaxf(bf16_lo(m2), bf16_hi(m2));
+                } else {
+                    zm = -CUDART_INF_F;
+#pragma unroll
+                    for (int u = 0; u < UNITS; ++u)
+                        zm = fmaxf(zm, fmaxf(fmaxf(__uint_as_float(raw[u].x), __uint_as_float(raw[u].y)),
+                                             fmaxf(__uint_as_float(raw[u].z), __uint_as_float(raw[u].w))));
+                }
+                new_reference(zm);
+#pragma unroll
+                for (int c = 0; c < PER / 8; ++c) {
+                    float z[8];
+                    if (DT == SPEC_BF16) {
+                        const uint4 r = raw[c];
+                        z[0] = bf16_lo(r.x); z[1] = bf16_hi(r.x); z[2] = bf16_lo(r.y); z[3] = bf16_hi(r.y);
+                        z[4] = bf16_lo(r.z); z[5] = bf16_hi(r.z); z[6] = bf16_lo(r.w); z[7] = bf16_hi(r.w);
+                    } else {
+                        const uint4 r0 = raw[c * NV], r1 = raw[c * NV + NV - 1];
+                        z[0] = __uint_as_float(r0.x); z[1] = __uint_as_float(r0.y); z[2] = __uint_as_float(r0.z); z[3] = __uint_as_float(r0.w);
+                        z[4] = __uint_as_float(r1.x); z[5] = __uint_as_float(r1.y); z[6] = __uint_as_float(r1.z); z[7] = __uint_as_float(r1.w);
+                    }
+                    add8(z);
+                }
+                flush();
+            }
+            cp_async_wait<0>();
+        }
+        // ---- the ragged end of the part, or every slice of a misaligned row: plain loads -----------------------
+        for (int t_base = (s_begin + nfull) * SLICE; t_base < tok_end; t_base += SLICE) {
+            const int n = min(SLICE, tok_end - t_base);
+            const unsigned char *src = rowp + (size_t)t_base * ESZ;
+            float z[PER];
+#pragma unroll
+            for (int c = 0; c < PER / 8; ++c) {
+                const int t0 = (tid + c * NT) * 8;
+                if (aligned && t0 + 8 <= n) {
+                    const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(tid + c * NT) * NV;
+                    if (DT == SPEC_BF16) {
+                        const uint4 r = __ldg(s4);
+                        z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
+                        z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
+                    } else {
+                        const uint4 r0 = __ldg(s4), r1 = __ldg(s4 + NV - 1);
+                        z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
+                        z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
+                }
+            }
+            float zm = -CUDART_INF_F;
+#pragma unroll
+            for (int k = 0; k < PER; ++k) zm = fmaxf(zm, z[k]);
+            new_reference(zm);
+#pragma unroll
+            for (int c = 0; c < PER / 8; ++c) {
+                float z8[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) z8[k] = z[c * 8 + k];
+                add8(z8);
+            }
+            flush();
         }
         // a NaN logit leaves a NaN in the sum; +inf was seen in the maximum
         bad |= !(fabsf(S_t) <= 3.0e38f);
-        cp_async_wait<0>();
         const int o_t = set ? (int)of : ROWPART_EMPTY;
 
         // ---- warp, then CTA: merge (reference, sums) pairs by exact powers of two --------------------------------

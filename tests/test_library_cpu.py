@@ -20,7 +20,7 @@ def lib():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "specverify.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\bint32_t\s+(spec_\w+)\s*\(", text)))
+    return sorted(set(re.findall(r"\bint(?:32|64)_t\s+(spec_\w+)\s*\(", text)))
 
 
 def test_every_declared_symbol_is_exported(lib):
