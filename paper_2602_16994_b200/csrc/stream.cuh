@@ -91,11 +91,14 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         const int b = (int)(row / P.N), a = (int)(row % P.N);
         RowPart *out = P.part + row2 * P.NSL + h;
         if (which == 1) {
-            // a draft row is read only for nodes that have children
+            // a draft row is read only for nodes that have children (every warp finds out by itself)
             const int *parent = P.parent + (long long)b * P.topo_stride;
             bool any = false;
-            for (int c = a + 1 + tid; c < P.N; c += NT) any |= __ldg(parent + c) == a;
-            if (!__syncthreads_or((int)any)) {
+            for (int c0 = a + 1; c0 < P.N && !any; c0 += 32) {
+                const int c = c0 + lane;
+                any = __any_sync(0xffffffffu, c < P.N && __ldg(parent + c) == a);
+            }
+            if (!any) {
                 if (tid == 0) { RowPart r = {}; r.O = ROWPART_EMPTY; r.cut = -CUDART_INF_F; r.bad = -1; *out = r; }
                 continue;
             }
@@ -182,6 +185,43 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
             };
 #pragma unroll
             for (int k = 0; k < DEPTH - 1; ++k) issue();
+            // ---- the ragged end of the part (and every slice of a misaligned row) by plain loads, while the ring fills
+            for (int t_base = (s_begin + nfull) * SLICE; t_base < tok_end; t_base += SLICE) {
+                const int n = min(SLICE, tok_end - t_base);
+                const unsigned char *src = rowp + (size_t)t_base * ESZ;
+                float z[PER];
+#pragma unroll
+                for (int c = 0; c < PER / 8; ++c) {
+                    const int t0 = (tid + c * NT) * 8;
+                    if (aligned && t0 + 8 <= n) {
+                        const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(tid + c * NT) * NV;
+                        if (DT == SPEC_BF16) {
+                            const uint4 r = __ldg(s4);
+                            z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
+                            z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
+                        } else {
+                            const uint4 r0 = __ldg(s4), r1 = __ldg(s4 + NV - 1);
+                            z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
+                            z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
+                    }
+                }
+                float zm = -CUDART_INF_F;
+#pragma unroll
+                for (int k = 0; k < PER; ++k) zm = fmaxf(zm, z[k]);
+                new_reference(zm);
+#pragma unroll
+                for (int c = 0; c < PER / 8; ++c) {
+                    float z8[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) z8[k] = z[c * 8 + k];
+                    add8(z8);
+                }
+                flush();
+            }
             for (int sl = 0; sl < nfull; ++sl) {
                 cp_async_wait<DEPTH - 2>();
                 const uint4 *st = ring + (size_t)cst * UNITS * NT + tid;
@@ -223,43 +263,6 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
             }
             cp_async_wait<0>();
         }
-        // ---- the ragged end of the part, or every slice of a misaligned row: plain loads -----------------------
-        for (int t_base = (s_begin + nfull) * SLICE; t_base < tok_end; t_base += SLICE) {
-            const int n = min(SLICE, tok_end - t_base);
-            const unsigned char *src = rowp + (size_t)t_base * ESZ;
-            float z[PER];
-#pragma unroll
-            for (int c = 0; c < PER / 8; ++c) {
-                const int t0 = (tid + c * NT) * 8;
-                if (aligned && t0 + 8 <= n) {
-                    const uint4 *s4 = reinterpret_cast<const uint4 *>(src) + (size_t)(tid + c * NT) * NV;
-                    if (DT == SPEC_BF16) {
-                        const uint4 r = __ldg(s4);
-                        z[c * 8 + 0] = bf16_lo(r.x); z[c * 8 + 1] = bf16_hi(r.x); z[c * 8 + 2] = bf16_lo(r.y); z[c * 8 + 3] = bf16_hi(r.y);
-                        z[c * 8 + 4] = bf16_lo(r.z); z[c * 8 + 5] = bf16_hi(r.z); z[c * 8 + 6] = bf16_lo(r.w); z[c * 8 + 7] = bf16_hi(r.w);
-                    } else {
-                        const uint4 r0 = __ldg(s4), r1 = __ldg(s4 + NV - 1);
-                        z[c * 8 + 0] = __uint_as_float(r0.x); z[c * 8 + 1] = __uint_as_float(r0.y); z[c * 8 + 2] = __uint_as_float(r0.z); z[c * 8 + 3] = __uint_as_float(r0.w);
-                        z[c * 8 + 4] = __uint_as_float(r1.x); z[c * 8 + 5] = __uint_as_float(r1.y); z[c * 8 + 6] = __uint_as_float(r1.z); z[c * 8 + 7] = __uint_as_float(r1.w);
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) z[c * 8 + k] = (t0 + k < n) ? load_logit(src, DT, t0 + k) : -CUDART_INF_F;
-                }
-            }
-            float zm = -CUDART_INF_F;
-#pragma unroll
-            for (int k = 0; k < PER; ++k) zm = fmaxf(zm, z[k]);
-            new_reference(zm);
-#pragma unroll
-            for (int c = 0; c < PER / 8; ++c) {
-                float z8[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) z8[k] = z[c * 8 + k];
-                add8(z8);
-            }
-            flush();
-        }
         // a NaN logit leaves a NaN in the sum; +inf was seen in the maximum
         bad |= !(fabsf(S_t) <= 3.0e38f);
         const int o_t = set ? (int)of : ROWPART_EMPTY;
@@ -269,29 +272,38 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         const int d = max(o_t - O_w, -100000);
         const double f = (double)pow2i(max(d, -127));
         const double Sw = warp_sum((double)S_t * f);
-        const double Xw = warp_sum(f * ((double)X_t + (double)d * (double)S_t));
-        double best = set ? (double)o_t + (double)xm_t : -1.0e300;
+        double Xw = 0.0, best = -1.0e300;
+        if (FEAT) {
+            Xw = warp_sum(f * ((double)X_t + (double)d * (double)S_t));
+            best = set ? (double)o_t + (double)xm_t : -1.0e300;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
+            for (int o = 16; o > 0; o >>= 1) best = fmax(best, __shfl_xor_sync(0xffffffffu, best, o));
+        }
         bad = __any_sync(0xffffffffu, bad);
         __syncthreads();             // the previous item's partials have been read
         if (lane == 0) { sS[w] = Sw; sX[w] = Xw; sB[w] = best; sO[w] = O_w; sBad[w] = bad; }
         __syncthreads();
-        if (tid == 0) {
-            int O = ROWPART_EMPTY, bd = 0;
-            double bst = -1.0e300;
-            for (int k = 0; k < NT / 32; ++k) { O = max(O, sO[k]); bd |= sBad[k]; bst = fmax(bst, sB[k]); }
-            double S = 0.0, X = 0.0;
-            for (int k = 0; k < NT / 32; ++k) {
-                const int dk = max(sO[k] - O, -100000);
-                const double fk = pow2d(dk);
-                S += sS[k] * fk;
-                X += fk * (sX[k] + (double)dk * sS[k]);
+        if (w == 0) {
+            // the warps' partials, one per lane
+            const bool has = lane < NT / 32;
+            const int Ok = has ? sO[lane] : ROWPART_EMPTY;
+            const int O = __reduce_max_sync(0xffffffffu, Ok);
+            const int dk = max(Ok - O, -100000);
+            const double fk = pow2d(dk), Sk = has ? sS[lane] : 0.0;
+            double S = Sk * fk, X = has ? fk * (sX[lane] + (double)dk * Sk) : 0.0, bst = has ? sB[lane] : -1.0e300;
+#pragma unroll
+            for (int o = (NT / 64); o > 0; o >>= 1) {
+                S += __shfl_xor_sync(0xffffffffu, S, o);
+                X += __shfl_xor_sync(0xffffffffu, X, o);
+                bst = fmax(bst, __shfl_xor_sync(0xffffffffu, bst, o));
             }
-            RowPart r;
-            r.S = S; r.X = X; r.O = O; r.xmax = O > ROWPART_EMPTY ? (float)(bst - (double)O) : 0.f;
-            r.cut = -CUDART_INF_F; r.bad = bd;
-            *out = r;
+            const int bd = __any_sync(0xffffffffu, has && sBad[lane]);
+            if (lane == 0) {
+                RowPart r;
+                r.S = S; r.X = X; r.O = O; r.xmax = (FEAT && O > ROWPART_EMPTY) ? (float)(bst - (double)O) : 0.f;
+                r.cut = -CUDART_INF_F; r.bad = bd;
+                *out = r;
+            }
         }
     }
 }
