@@ -15,6 +15,7 @@
 #include "cut.cuh"
 #include "rowops.cuh"
 #include "rowstat.cuh"
+#include "tree.cuh"
 #include "specverify.h"
 #include "verify.cuh"
 #include "walk.cuh"
@@ -154,7 +155,8 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 struct WsLayout {
     int64_t rec, pub, done, cut, stat, clear_bytes, total;
 };
-WsLayout ws_layout(const SpecIn *in, int slices = 32)   // slices = 0: merged rows only
+constexpr int MAX_PARTS = 4;      // parts a row may be split into by the streaming statistics kernel
+WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: one record per row only
 {
     WsLayout L;
     const int64_t nodes = (int64_t)in->B * in->N;
@@ -165,7 +167,7 @@ WsLayout ws_layout(const SpecIn *in, int slices = 32)   // slices = 0: merged ro
     L.clear_bytes = o - L.pub;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
-    L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // merged rows, then slices
+    L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // one record per row, then the parts
     L.total = o;
     return L;
 }
@@ -272,18 +274,18 @@ int resident_clusters(K kernel, int C, int threads, int smem)
     return n;
 }
 
-template <int DT, int NW, bool FEAT>
-int launch_verify(const VPlan &pl, VParams &vp, cudaStream_t st)
+template <int DT, int NW>
+int launch_tree(const VPlan &pl, TParams &tp, cudaStream_t st)
 {
-    auto kernel = spec_verify_kernel<DT, NW, FEAT>;
+    auto kernel = spec_tree_kernel<DT, NW>;
     int rc = prepare_kernel(kernel, pl.C, pl.smem);
     if (rc) return rc;
     const int threads = (NW + 1) * 32;
     int nc = resident_clusters(kernel, pl.C, threads, pl.smem);
     if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
-    const long long nodes = (long long)vp.B * vp.N;
+    const long long nodes = (long long)tp.v.B * tp.v.N;
     if (nc > nodes) nc = (int)nodes;
-    return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &vp);
+    return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &tp);
 }
 
 // row statistics (cut, reference, normaliser) of every row the verifiers read, or of every row of `z`
@@ -335,8 +337,11 @@ int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
     return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &wp);
 }
 
-int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl,
-                bool trunc, cudaStream_t st)
+// Statistics of every row the verifiers read (reference, normaliser, cut; one record per row at the
+// start of the statistics region), and the entropy features when asked for.  `parts`: the streaming
+// kernel may split rows into parts (needs the parts region of the workspace).
+int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, bool trunc, bool parts,
+                   cudaStream_t st)
 {
     int rc;
     int NSL = 1;
@@ -349,7 +354,7 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         const long long rows2 = 2ll * in->B * in->N;
         const int slices_row = (in->V + stream::SLICE - 1) / stream::SLICE;
         NSL = 1;
-        while (NSL < 4 && NSL < slices_row && rows2 * NSL < 2 * sm_count()) NSL *= 2;
+        while (parts && NSL < MAX_PARTS && NSL < slices_row && rows2 * NSL < 2 * sm_count()) NSL *= 2;
         stream::SParams sp = {};
         sp.B = in->B; sp.N = in->N; sp.V = in->V; sp.NSL = NSL;
         sp.zp = in->target_logits; sp.zq = in->draft_logits;
@@ -388,6 +393,16 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
         g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     }
+    return SPEC_OK;
+}
+
+int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl,
+                bool trunc, cudaStream_t st)
+{
+    int rc = row_statistics(in, out, w, L, trunc, true, st);
+    if (rc) return rc;
+    const int NSL = 1;
+    RowPart *part = (RowPart *)(w + L.stat);
     WParams wp = {};
     wp.B = in->B; wp.N = in->N; wp.V = in->V; wp.C = pl.C; wp.NSL = NSL;
     wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.off_x = pl.off_x; wp.off_es = pl.off_es; wp.off_ring = pl.off_ring;
@@ -401,14 +416,14 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
 }
 
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode,
-                  bool allow_walk = true)
+                  bool allow_walk = true, bool parts = true)
 {
     int rc = check_in(in, true);
     if (rc) return rc;
     if (!out || !out->accepted_node || !out->accept_len || !out->out_tokens || !out->bonus_token || !out->status)
         return SPEC_ERR_NULL;
     const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
-    const WsLayout L = ws_layout(in);
+    const WsLayout L = ws_layout(in, parts ? MAX_PARTS : 0);
     if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
     VPlan pl;
     if (!make_vplan(in->V, in->logits_dtype, &pl)) return SPEC_ERR_UNSUPPORTED;
@@ -431,11 +446,11 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         cudaGetLastError();
         return SPEC_ERR_CUDA;
     }
-    if (trunc) {
-        rc = launch_rowstat(in, in->target_logits, in->draft_logits, in->parent, w, L, st);
-        if (rc) return rc;
-    }
-    VParams vp = {};
+    // every node of every sequence on chip once, on top of the row statistics
+    rc = row_statistics(in, out, w, L, trunc, parts, st);
+    if (rc) return rc;
+    TParams tp = {};
+    VParams &vp = tp.v;
     vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
     vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
     vp.slice_len = pl.slice_len; vp.NS = pl.NS;
@@ -444,22 +459,17 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
     vp.parent = in->parent; vp.token = in->token;
     vp.T = in->temperature; vp.T_seq = in->temperature_per_seq;
-    vp.cut = trunc ? (const float *)(w + L.cut) : nullptr;
+    vp.cut = nullptr;
     vp.u_accept = in->u_accept; vp.u_bonus = in->u_bonus;
     vp.rec = (NodeRec *)(w + L.rec);
     vp.w_pub = (unsigned long long *)(w + L.pub);
     vp.done = (unsigned int *)(w + L.done);
-    vp.features = out->node_features;
+    vp.features = nullptr;
     vp.out = *out;
-    const bool feat = out->node_features != nullptr;
+    tp.part = (const RowPart *)(w + L.stat);
     const bool bf = in->logits_dtype == SPEC_BF16;
-    if (pl.NW == 7) {
-        if (bf) rc = feat ? launch_verify<SPEC_BF16, 7, true>(pl, vp, st) : launch_verify<SPEC_BF16, 7, false>(pl, vp, st);
-        else rc = feat ? launch_verify<SPEC_F32, 7, true>(pl, vp, st) : launch_verify<SPEC_F32, 7, false>(pl, vp, st);
-    } else {
-        if (bf) rc = feat ? launch_verify<SPEC_BF16, 15, true>(pl, vp, st) : launch_verify<SPEC_BF16, 15, false>(pl, vp, st);
-        else rc = feat ? launch_verify<SPEC_F32, 15, true>(pl, vp, st) : launch_verify<SPEC_F32, 15, false>(pl, vp, st);
-    }
+    if (pl.NW == 7) rc = bf ? launch_tree<SPEC_BF16, 7>(pl, tp, st) : launch_tree<SPEC_F32, 7>(pl, tp, st);
+    else rc = bf ? launch_tree<SPEC_BF16, 15>(pl, tp, st) : launch_tree<SPEC_F32, 15>(pl, tp, st);
     if (rc) return rc;
     if (out->residual) {
         RParams rp = {};
@@ -584,7 +594,7 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
     void *ws = nullptr;
     rc = static_ws_address(&ws);
     if (rc) return rc;
-    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false);
+    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false, false);
 }
 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,

@@ -1,0 +1,510 @@
+// Whole-tree verification on top of the row statistics (stream.cuh / rowstat.cuh): every node of
+// every sequence is one work item of a thread-block cluster, as Traversal Verification needs (its
+// weights are defined for every node, top-down: Section 3.2) and as SpecInfer's diagnostic outputs
+// need (the threshold of every node, Algorithm 4).
+//
+// With a row's reference O and normaliser Z known before the node comes on chip, a node is:
+//   scalars   children, their tokens and uniforms, the final probabilities p(x_c), q(x_c) of every
+//             child's token (two logits and two normalisers each) -- loaded while the producer
+//             warp's bulk copies of the node's rows are in flight;
+//   pass 1    e = 2^(z s - O) of both rows, resident in registers and shared memory, all threads in
+//             the same units (no per-thread references, no exchange of normalisers);
+//   weight    Traversal: the weight the parent published for this node (bounded poll);
+//   siblings  the residual recursion  U_j = (w_in P0 - c_j q)+,  c_{j+1} = c_j + G_j,
+//             E_j = sum U_j,  G_{j+1} = E_{j+1} + G_j - E_j  (SpecInfer: w_in = 1, G = E), one pass
+//             over the resident e and one distributed-shared-memory exchange per rejected child;
+//             child j is handed min(1, U_j(x_j) / (G_j q(x_j))), published at once;
+//   outcome   w_fin = E / G; where the node can be the accepted one, the bonus token by an
+//             inverse-CDF search over the committed residual.
+// Records, published weights, arrival counting and the writing of a sequence's outputs are those of
+// verify.cuh.
+#pragma once
+#include "stream.cuh"
+#include "verify.cuh"
+
+namespace specv {
+
+struct TParams {
+    VParams v;                // shapes, inputs, records, published weights, arrival counters, outputs
+    const RowPart *part;      // [B*N*2] statistics of every row the verifier reads
+};
+
+template <int DT, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kernel(const TParams TP)
+{
+    const VParams &P = TP.v;
+    constexpr bool FEAT = false;
+    constexpr int NCONS = NW * 32;
+    constexpr int TILE = NCONS * 8;
+    constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
+    constexpr int ROWB = TILE * ESZ;
+    constexpr int STAGE = 2 * ROWB;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    Hdr &S = *reinterpret_cast<Hdr *>(dyn_smem);
+    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW]
+    float4 *es = reinterpret_cast<float4 *>(dyn_smem + P.off_es);    // [slot][p lo, p hi, q lo, q hi][NCONS]
+    unsigned char *ring = dyn_smem + P.off_ring;
+    const int C = P.C, NS = P.NS;
+    const unsigned rank = cluster_ctarank();
+    const int cid = blockIdx.x / C, NC = gridDim.x / C;
+    const long long total = (long long)P.B * P.N;
+    const long long tok0 = (long long)rank * P.slice_len;
+    const int n_slice = (int)max(0ll, min((long long)P.slice_len, (long long)P.V - tok0));
+    const int ntiles = (n_slice + TILE - 1) / TILE;
+    const int nsm = max(ntiles - RT, 0), nrg = ntiles - nsm;
+    const bool trav = P.mode == MODE_TRAVERSAL;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], NW); }
+        mbar_init(&S.xbar[0], 1);
+        mbar_init(&S.xbar[1], 1);
+        S.poison = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    cluster_sync_all();
+
+    if (warp == NW) {
+        // ======================= producer warp: fills the ring, node after node =======================
+        int g = 0;
+        bool ok = true;
+        for (long long id = cid; id < total && ok; id += NC) {
+            const int a = (int)(id / P.B), b = (int)(id % P.B);
+            const bool hq = warp_has_children(P.parent + (long long)b * P.topo_stride, P.N, a, lane);
+            const long long row = (long long)b * P.seq_stride + (long long)a * P.node_stride + tok0;
+            const unsigned char *src_p = (const unsigned char *)P.zp + row * ESZ;
+            const unsigned char *src_q = (const unsigned char *)P.zq + row * ESZ;
+            const bool aligned = ((((uintptr_t)src_p) | (hq ? (uintptr_t)src_q : 0)) & 15) == 0;
+            for (int i = 0; i < ntiles; ++i, ++g) {
+                const int stage = g % NS, use = g / NS;
+                if (use > 0) {
+                    int w = 1;
+                    if (lane == 0) w = mbar_wait(&S.empty[stage], (uint32_t)((use - 1) & 1)) ? 1 : 0;
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w || *(volatile int *)&S.poison) { S.poison = 1; ok = false; break; }
+                }
+                const int ntok = min(TILE, n_slice - i * TILE);
+                unsigned char *dst_p = ring + (size_t)stage * STAGE, *dst_q = dst_p + ROWB;
+                const unsigned char *sp = src_p + (size_t)i * ROWB, *sq = src_q + (size_t)i * ROWB;
+                const uint32_t body = aligned ? (((uint32_t)ntok * ESZ) & ~15u) : 0u;
+                // what the bulk copy cannot take (a misaligned row, the last few bytes): plain loads
+                if (ESZ == 2) {
+                    for (int e = (int)(body / 2) + lane; e < ntok; e += 32) {
+                        ((unsigned short *)dst_p)[e] = __ldg((const unsigned short *)sp + e);
+                        if (hq) ((unsigned short *)dst_q)[e] = __ldg((const unsigned short *)sq + e);
+                    }
+                } else {
+                    for (int e = (int)(body / 4) + lane; e < ntok; e += 32) {
+                        ((float *)dst_p)[e] = __ldg((const float *)sp + e);
+                        if (hq) ((float *)dst_q)[e] = __ldg((const float *)sq + e);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    if (body) {
+                        mbar_arrive_expect_tx(&S.full[stage], hq ? 2 * body : body);
+                        bulk_g2s(dst_p, sp, body, &S.full[stage]);
+                        if (hq) bulk_g2s(dst_q, sq, body, &S.full[stage]);
+                    } else {
+                        mbar_arrive(&S.full[stage]);
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            // gave up: wait (bounded) for the copies still in flight before leaving
+            for (int k = 1; k <= NS && k <= g; ++k) {
+                const int gg = g - k;
+                mbar_wait(&S.full[gg % NS], (uint32_t)((gg / NS) & 1));
+            }
+        }
+    } else {
+        // ================================ consumer warps ================================================
+        WarpArea &W = S.wa[warp];
+        const bool scribe = rank == 0 && warp == 0;     // the one warp that writes the node's record
+        int stage = 0;
+        uint32_t phase = 0;
+        int xn = 0;
+        float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
+
+        for (long long id = cid; id < total; id += NC) {
+            const int a = (int)(id / P.B), b = (int)(id % P.B);
+            const int *parent = P.parent + (long long)b * P.topo_stride;
+            const int *token = P.token + (long long)b * P.N;
+            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+            float s_hi = (float)s_d;
+            if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
+            float s_lo = (float)(s_d - (double)s_hi);
+            if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
+
+            // ---- the node's scalars (the producer's copies are in flight meanwhile) ---------------------------
+            int kc = 0, err = 0;
+            if (lane == 0) {
+                const int pa = __ldg(parent + a);
+                if (a == 0 ? (pa != -1) : (pa < 0 || pa >= a)) err = SPEC_DEV_TOPOLOGY;
+                if (a > 0) {
+                    const int x = __ldg(token + a);
+                    if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                }
+            }
+            for (int c0 = a + 1; c0 < P.N; c0 += 32) {
+                const int c = c0 + lane;
+                const bool is = c < P.N && __ldg(parent + c) == a;
+                const unsigned bal = __ballot_sync(0xffffffffu, is);
+                if (is) {
+                    const int pos = kc + __popc(bal & ((1u << lane) - 1u));
+                    if (pos < KMAX) {
+                        const int x = __ldg(token + c);
+                        W.child[pos] = c;
+                        W.cpn[pos] = x;
+                        W.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
+                        if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                    }
+                }
+                kc += __popc(bal);
+            }
+            if (kc > KMAX) err = SPEC_DEV_TOPOLOGY;
+            const bool hq = kc > 0;
+            // statistics of the node's rows
+            const RowPart *rp = TP.part + ((long long)b * P.N + a) * 2;
+            const double Z_p = __ldcg(&rp[0].S);
+            const int O_p = __ldcg(&rp[0].O);
+            const float cut_p = __ldcg(&rp[0].cut);
+            double Z_q = 0.0;
+            int O_q = ROWPART_EMPTY;
+            float cut_q = -CUDART_INF_F;
+            bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
+            if (hq) {
+                Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
+                bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
+            }
+            err = __reduce_max_sync(0xffffffffu, err);
+            if (bad && !err) err = SPEC_DEV_NONFINITE;
+            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
+            // final probabilities of the children's tokens (lanes j: target, 16 + j: draft)
+            __syncwarp();
+            {
+                const int j = lane & 15;
+                const bool mine = !err && j < kc;
+                const int xt = mine ? W.cpn[j] : 0;
+                __syncwarp();
+                if (mine) {
+                    const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
+                    const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + xt);
+                    const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
+                    double pr = 0.0;
+                    if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
+                        const double nd = rint(xd);
+                        pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
+                    }
+                    if (lane < 16) W.cpm[j] = pr; else W.cqm[j] = pr;
+                }
+                __syncwarp();
+            }
+
+            // ---- pass 1: e = 2^(z s - O) of both rows, resident ------------------------------------------------
+            bool poisoned = *(volatile int *)&S.poison != 0;
+            {
+                const float ofp = (float)O_p, ofq = (float)O_q;
+                RawChunk<DT> raw_p, raw_q;
+                float z[8];
+                float dsx = 0.f;
+#define SPECT_NEXT_TILE(TILE_INDEX)                                                                          \
+                if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; }       \
+                {                                                                                            \
+                    const unsigned char *sp_ = ring + (size_t)stage * STAGE + (size_t)tid * 8 * ESZ;         \
+                    raw_p = read_raw<DT>(sp_);                                                               \
+                    if (hq) raw_q = read_raw<DT>(sp_ + ROWB);                                                \
+                }                                                                                            \
+                __syncwarp();                                                                                \
+                if (lane == 0) mbar_arrive(&S.empty[stage]);                                                 \
+                if (++stage == NS) { stage = 0; phase ^= 1u; }                                               \
+                const int nvalid = poisoned ? 0 : n_slice - ((TILE_INDEX) * TILE + tid * 8);
+                for (int i = 0; i < nsm; ++i) {
+                    SPECT_NEXT_TILE(i)
+                    float e8[8];
+                    unpack_chunk<DT>(raw_p, z);
+                    mask_chunk(z, nvalid, true, cut_p);
+                    exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
+                    float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                    d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
+                    d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
+                    if (hq) {
+                        unpack_chunk<DT>(raw_q, z);
+                        mask_chunk(z, nvalid, true, cut_q);
+                        exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
+                        d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
+                        d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
+                    } else {
+                        d[2 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        d[3 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+#define SPECT_REG_TILE(J, EP, EQ)                                                                            \
+                if ((J) < nrg) {                                                                             \
+                    SPECT_NEXT_TILE(nsm + (J))                                                               \
+                    unpack_chunk<DT>(raw_p, z);                                                              \
+                    mask_chunk(z, nvalid, true, cut_p);                                                      \
+                    exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                            \
+                    if (hq) {                                                                                \
+                        unpack_chunk<DT>(raw_q, z);                                                          \
+                        mask_chunk(z, nvalid, true, cut_q);                                                  \
+                        exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                        \
+                    } else {                                                                                 \
+                        _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                           \
+                    }                                                                                        \
+                } else {                                                                                     \
+                    _Pragma("unroll") for (int k = 0; k < 8; ++k) { EP[k] = 0.f; EQ[k] = 0.f; }              \
+                }
+                SPECT_REG_TILE(0, ep0, eq0)
+                SPECT_REG_TILE(1, ep1, eq1)
+                SPECT_REG_TILE(2, ep2, eq2)
+                SPECT_REG_TILE(3, ep3, eq3)
+#undef SPECT_REG_TILE
+#undef SPECT_NEXT_TILE
+            }
+            if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
+
+            // ---- Traversal: the weight handed down by the parent (bounded poll, every warp for itself) ------
+            double w_in = 1.0;
+            if (trav && a > 0 && !err) {
+                unsigned long long bits = W_PENDING;
+                if (lane == 0) {
+                    volatile unsigned long long *slot = P.w_pub + (long long)b * P.N + a;
+                    const long long t0 = clock64();
+                    for (;;) {
+                        bits = *slot;
+                        if (bits != W_PENDING || clock64() - t0 > WAIT_CYCLES || *(volatile int *)&S.poison) break;
+                        __nanosleep(32);
+                    }
+                    __threadfence();
+                }
+                bits = __shfl_sync(0xffffffffu, bits, 0);
+                if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
+                else w_in = __longlong_as_double((long long)bits);
+            }
+
+            // ---- state of the recursion (identical in every warp of the cluster) ------------------------------
+            const bool live = !err && w_in > 0.0;
+            const double A = live ? w_in * invZp : 0.0;
+            const double Rg = (live && hq) ? Z_p * invZq * (w_in == 1.0 ? 1.0 : __drcp_rn(w_in)) : 0.0;
+            double st_c = 0.0, st_E = err ? 0.0 : w_in, st_G = 1.0, g_commit = 0.0;
+            double E_r = 0.0;            // lane r: rank r's total of the committed U
+            bool have_E = false;
+
+            // one pass over the resident e with coefficient g, then the exchange: lane r gets rank r's
+            // total in y, every lane the cluster's total (bit-identical in every warp of the cluster)
+            auto pass = [&](double g, double &y) -> double {
+                float g_hi, g_lo;
+                split_float(g, g_hi, g_lo);
+                float tot = 0.f;
+                for (int i = 0; i < nsm; ++i) {
+                    float p[8], q[8];
+                    const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                    load_e8(d, NCONS, p);
+                    load_e8(d + 2 * NCONS, NCONS, q);
+                    tot += residual_chunk(p, q, g_hi, g_lo);
+                }
+                tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
+                       (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
+                const double wsum = A * warp_sum((double)tot);
+                const int par = xn & 1;
+                if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
+                if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
+                if (!*(volatile int *)&S.poison && !mbar_wait_cluster(&S.xbar[par], (uint32_t)((xn >> 1) & 1))) S.poison = 1;
+                ++xn;
+                y = 0.0;
+                if (lane < C) {
+                    const double *src = xchg + (size_t)(par * C + lane) * NW;
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) y += src[w];
+                }
+                return warp_sum(y);
+            };
+
+            bool dead = !(A > 0.0);
+            int acc = -1;
+            const int kce = min(kc, KMAX);
+            if (err && scribe && lane == 0) {
+                // nothing below a faulty node is evaluated: every child gets weight / threshold 0
+                NodeRec *rec = P.rec + (long long)b * P.N;
+                for (int c = a + 1; c < P.N; ++c)
+                    if (__ldg(parent + c) == a) {
+                        if (trav) {
+                            rec[c].w_in = 0.0;
+                            __threadfence();
+                            *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
+                        } else {
+                            rec[c].thr = 0.0;
+                        }
+                    }
+            }
+            for (int j = 0; j < kce && !err; ++j) {
+                const double Pp = W.cpm[j], Pq = W.cqm[j];
+                const double Ux = w_in * Pp - st_c * Pq;
+                const double denom = trav ? st_G : st_E;
+                const bool zero = dead || !(Ux > 0.0), one = !zero && !(Pq > 0.0);
+                if (scribe) {
+                    const double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
+                    if (lane == 0) {
+                        NodeRec *rec = P.rec + (long long)b * P.N;
+                        const int cj = W.child[j];
+                        if (trav) {
+                            rec[cj].w_in = thr;
+                            __threadfence();
+                            *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
+                                (unsigned long long)__double_as_longlong(thr);
+                        } else {
+                            rec[cj].thr = thr;
+                        }
+                    }
+                }
+                if (!trav && acc < 0 && !zero && (one || (double)W.cu[j] * denom * Pq < Ux)) {
+                    acc = W.child[j];
+                    if (!P.all_thr) {
+                        if (scribe && lane == 0)
+                            for (int jj = j + 1; jj < kce; ++jj) P.rec[(long long)b * P.N + W.child[jj]].thr = CUDART_NAN;
+                        break;
+                    }
+                }
+                if (dead) continue;          // weight 0: the remaining children need no pass
+                // residual step after rejecting child j: c' = c + G
+                const double g = (st_c + st_G) * Rg;
+                double y;
+                const double En = pass(g, y);
+                if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
+                if (En > 0.0) {
+                    const double c_new = st_c + st_G, G_new = En + st_G - st_E;
+                    st_c = c_new; st_G = G_new; st_E = En;
+                    g_commit = g;
+                    E_r = y;
+                    have_E = true;
+                } else if (!(st_E >= st_G)) {
+                    dead = true;       // S = 0 with w < 1: the weight drops to 0 (Traversal only)
+                    st_E = 0.0;
+                }
+                // else S = 0 with w = 1 (P equals q up to rounding): the state stays
+            }
+
+            // ---- the node's outcome -----------------------------------------------------------------------------
+            const double w_fin = (dead || err) ? 0.0 : st_E / st_G;
+            bool want_bonus;
+            if (trav) want_bonus = (a == 0) || ((double)__ldg(P.u_accept + (long long)b * P.N + a) < w_fin);
+            else want_bonus = acc < 0;
+            if (dead || err) want_bonus = false;
+            int owner = -1;
+            double tau = 0.0, E_tot = 0.0;
+            if (want_bonus) {
+                if (!have_E) {
+                    // no residual step was taken: the totals of U_0 = w_in P0 per rank
+                    pass(0.0, E_r);
+                    if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; want_bonus = false; }
+                }
+            }
+            if (want_bonus) {
+                E_tot = warp_sum(lane < C ? E_r : 0.0);
+                const double target = (double)__ldg(P.u_bonus + (long long)b * P.N + a) * E_tot;
+                owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
+            }
+            if (scribe) {
+                if (lane == 0) {
+                    NodeRec &R = P.rec[(long long)b * P.N + a];
+                    R.O_p = (double)O_p; R.Z_p = Z_p; R.O_q = (double)O_q; R.Z_q = Z_q;
+                    R.c_fin = st_c; R.E_fin = (dead || err) ? 0.0 : st_E;
+                    R.cut_p = cut_p; R.cut_q = cut_q;
+                    R.next_child = acc;
+                    R.status = err;
+                    if (trav) { R.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) R.w_in = 1.0; }
+                    else { R.w_in = 1.0; if (a == 0) R.thr = 1.0; }
+                    if (owner < 0) { R.bonus = -1; R.bonus_margin = 0.f; }
+                }
+                arrive_sequence(P, b, owner < 0 ? 2u : 1u);
+            }
+
+            // ---- bonus token: inverse CDF over the owner CTA's slice -----------------------------------------
+            if (owner == (int)rank) {
+                float gh_c, gl_c;
+                split_float(g_commit, gh_c, gl_c);
+                const double invA = 1.0 / A;
+                const double tau_rel = tau * invA, tot_rel = E_tot * invA;       // in units of e
+                for (int i = 0; i < nsm; ++i) {
+                    float p[8], q[8];
+                    const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+                    load_e8(d, NCONS, p);
+                    load_e8(d + 2 * NCONS, NCONS, q);
+                    const double r = warp_sum((double)residual_chunk(p, q, gh_c, gl_c));
+                    if (lane == 0) S.wtile[warp][i] = r;
+                }
+                {
+                    const double r0 = warp_sum((double)residual_chunk(ep0, eq0, gh_c, gl_c));
+                    const double r1 = warp_sum((double)residual_chunk(ep1, eq1, gh_c, gl_c));
+                    const double r2 = warp_sum((double)residual_chunk(ep2, eq2, gh_c, gl_c));
+                    const double r3 = warp_sum((double)residual_chunk(ep3, eq3, gh_c, gl_c));
+                    if (lane == 0) {
+                        S.wtile[warp][nsm] = r0; S.wtile[warp][nsm + 1] = r1;
+                        S.wtile[warp][nsm + 2] = r2; S.wtile[warp][nsm + 3] = r3;
+                    }
+                }
+                bar_sync(1, NCONS);
+                // tile, then warp inside the tile, then lane inside the warp, then token inside the chunk
+                double Ti = 0.0;
+                if (lane < nsm + RT)
+                    for (int w = 0; w < NW; ++w) Ti += S.wtile[w][lane];
+                double tau2, tau3, tau4;
+                const int i_star = pick_lane(Ti, tau_rel, tau2);
+                const double Ww = (i_star >= 0 && lane < NW) ? S.wtile[lane][i_star] : 0.0;
+                const int w_star = i_star >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
+                bar_sync(1, NCONS);          // wtile may be rewritten by the next node only after everyone has read it
+                if (w_star < 0) {
+                    if (warp == 0) {
+                        if (lane == 0) { NodeRec &R = P.rec[(long long)b * P.N + a]; R.bonus = -1; R.bonus_margin = 0.f; }
+                        arrive_sequence(P, b, 1u);
+                    }
+                } else if (warp == w_star) {
+                    float p[8], q[8];
+                    if (i_star < nsm) {
+                        const float4 *d = es + (size_t)(i_star * 4) * NCONS + tid;
+                        load_e8(d, NCONS, p);
+                        load_e8(d + 2 * NCONS, NCONS, q);
+                    } else {
+                        const int jr = i_star - nsm;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
+                            q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
+                        }
+                    }
+                    float wk[8], v = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl_c, q[k], fmaf(-gh_c, q[k], p[k])), 0.f); v += wk[k]; }
+                    const int l_star = pick_lane((double)v, tau3, tau4);
+                    if (lane == l_star) {
+                        double run = 0.0, dlo = 0.0, dhi = 0.0;
+                        int found = -1, last_pos = -1;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const double before = run;
+                            run += (double)wk[k];
+                            if (wk[k] > 0.f) last_pos = k;
+                            if (found < 0 && run > tau4) { found = k; dlo = tau4 - before; dhi = run - tau4; }
+                        }
+                        if (found < 0) { found = last_pos; dlo = 0.0; dhi = 0.0; }
+                        NodeRec &R = P.rec[(long long)b * P.N + a];
+                        R.bonus = found >= 0 ? (int)(tok0 + (long long)i_star * TILE + tid * 8 + found) : -1;
+                        R.bonus_margin = (float)(fmin(dlo, dhi) / tot_rel);
+                    } else if (l_star < 0 && lane == 0) {
+                        NodeRec &R = P.rec[(long long)b * P.N + a];
+                        R.bonus = -1;
+                        R.bonus_margin = 0.f;
+                    }
+                    __syncwarp();
+                    arrive_sequence(P, b, 1u);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    cluster_sync_all();        // nobody leaves while a peer may still write to its shared memory
+}
+
+}  // namespace specv
