@@ -5,8 +5,8 @@
 //
 // With a row's reference O and normaliser Z known before the node comes on chip, a node is:
 //   scalars   children, their tokens and uniforms, the final probabilities p(x_c), q(x_c) of every
-//             child's token (two logits and two normalisers each) -- loaded while the producer
-//             warp's bulk copies of the node's rows are in flight;
+//             child's token (two logits and two normalisers each) -- gathered by the producer warp,
+//             one node ahead of the consumers, into a double-buffered block of shared memory;
 //   pass 1    e = 2^(z s - O) of both rows, resident in registers and shared memory, all threads in
 //             the same units (no per-thread references, no exchange of normalisers);
 //   weight    Traversal: the weight the parent published for this node (bounded poll);
@@ -29,6 +29,25 @@ struct TParams {
     const RowPart *part;      // [B*N*2] statistics of every row the verifier reads
 };
 
+// what the consumers need to know about a node besides its rows
+struct __align__(16) NodeScalars {
+    double Z_p, Z_q;
+    double cpm[KMAX], cqm[KMAX];   // final probabilities of the children's tokens under p and q
+    float cu[KMAX];                // the children's acceptance uniforms
+    int child[KMAX];
+    int kc, err, O_p, O_q;
+    float cut_p, cut_q, u_a, ub_a;
+};
+
+struct __align__(16) THdr {
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], sfull[2], sempty[2];
+    double wtile[NWMAX + 1][TMAX];
+    NodeScalars sc[2];
+    int poison;
+};
+
+static_assert(sizeof(THdr) <= sizeof(Hdr), "the launch plan reserves sizeof(Hdr) bytes for the header");
+
 template <int DT, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kernel(const TParams TP)
 {
@@ -40,7 +59,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     constexpr int ROWB = TILE * ESZ;
     constexpr int STAGE = 2 * ROWB;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    Hdr &S = *reinterpret_cast<Hdr *>(dyn_smem);
+    THdr &S = *reinterpret_cast<THdr *>(dyn_smem);
     double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW]
     float4 *es = reinterpret_cast<float4 *>(dyn_smem + P.off_es);    // [slot][p lo, p hi, q lo, q hi][NCONS]
     unsigned char *ring = dyn_smem + P.off_ring;
@@ -58,6 +77,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         for (int s = 0; s < NS; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], NW); }
         mbar_init(&S.xbar[0], 1);
         mbar_init(&S.xbar[1], 1);
+        mbar_init(&S.sfull[0], 1);
+        mbar_init(&S.sfull[1], 1);
+        mbar_init(&S.sempty[0], NW);
+        mbar_init(&S.sempty[1], NW);
         S.poison = 0;
         mbar_fence_init();
     }
@@ -65,10 +88,99 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     cluster_sync_all();
 
     if (warp == NW) {
-        // ======================= producer warp: fills the ring, node after node =======================
+        // ======================= producer warp: fills the ring, node after node, and gathers the =======
+        // ======================= scalars of the node after the one whose rows it has just issued =======
         int g = 0;
         bool ok = true;
-        for (long long id = cid; id < total && ok; id += NC) {
+        // scalars of item `id` (the kidx-th item of this cluster) into block kidx & 1
+        auto scalars = [&](long long id, int kidx) {
+            const int a = (int)(id / P.B), b = (int)(id % P.B);
+            const int buf = kidx & 1;
+            if (kidx >= 2) {
+                int w = 1;
+                if (lane == 0) w = mbar_wait(&S.sempty[buf], (uint32_t)(((kidx >> 1) - 1) & 1)) ? 1 : 0;
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w || *(volatile int *)&S.poison) { S.poison = 1; ok = false; return; }
+            }
+            NodeScalars &N = S.sc[buf];
+            const int *parent = P.parent + (long long)b * P.topo_stride;
+            const int *token = P.token + (long long)b * P.N;
+            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+            int kc = 0, err = 0;
+            if (lane == 0) {
+                const int pa = __ldg(parent + a);
+                if (a == 0 ? (pa != -1) : (pa < 0 || pa >= a)) err = SPEC_DEV_TOPOLOGY;
+                if (a > 0) {
+                    const int x = __ldg(token + a);
+                    if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                }
+                N.u_a = __ldg(P.u_accept + (long long)b * P.N + a);
+                N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
+            }
+            int my_tok = 0;              // lanes j and 16 + j: token of child j
+            for (int c0 = a + 1; c0 < P.N; c0 += 32) {
+                const int c = c0 + lane;
+                const bool is = c < P.N && __ldg(parent + c) == a;
+                const unsigned bal = __ballot_sync(0xffffffffu, is);
+                if (is) {
+                    const int pos = kc + __popc(bal & ((1u << lane) - 1u));
+                    if (pos < KMAX) {
+                        const int x = __ldg(token + c);
+                        N.child[pos] = c;
+                        N.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
+                        N.cpm[pos] = (double)x;          // parked here until the probabilities are known
+                        if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                    }
+                }
+                kc += __popc(bal);
+            }
+            if (kc > KMAX) err = SPEC_DEV_TOPOLOGY;
+            const bool hq = kc > 0;
+            const RowPart *rp = TP.part + ((long long)b * P.N + a) * 2;
+            const double Z_p = __ldcg(&rp[0].S);
+            const int O_p = __ldcg(&rp[0].O);
+            const float cut_p = __ldcg(&rp[0].cut);
+            double Z_q = 0.0;
+            int O_q = ROWPART_EMPTY;
+            float cut_q = -CUDART_INF_F;
+            bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
+            if (hq) {
+                Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
+                bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
+            }
+            err = __reduce_max_sync(0xffffffffu, err);
+            if (bad && !err) err = SPEC_DEV_NONFINITE;
+            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
+            __syncwarp();
+            {
+                const int j = lane & 15;
+                const bool mine = !err && j < kc;
+                my_tok = mine ? (int)N.cpm[j] : 0;
+                __syncwarp();
+                double pr = 0.0;
+                if (mine) {
+                    const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
+                    const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + my_tok);
+                    const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
+                    if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
+                        const double nd = rint(xd);
+                        pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
+                    }
+                }
+                if (j < KMAX) { if (lane < 16) N.cpm[j] = pr; else N.cqm[j] = pr; }
+            }
+            if (lane == 0) {
+                N.Z_p = Z_p; N.Z_q = Z_q; N.O_p = O_p; N.O_q = O_q; N.cut_p = cut_p; N.cut_q = cut_q;
+                N.kc = kc; N.err = err;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.sfull[buf]);
+        };
+        // pass 1 needs a node's references and cuts, so its scalars come before its rows: the first
+        // node's before anything else, from then on one node ahead
+        int kidx = 0;
+        if (cid < total) scalars(cid, 0);
+        for (long long id = cid; id < total && ok; id += NC, ++kidx) {
             const int a = (int)(id / P.B), b = (int)(id % P.B);
             const bool hq = warp_has_children(P.parent + (long long)b * P.topo_stride, P.N, a, lane);
             const long long row = (long long)b * P.seq_stride + (long long)a * P.node_stride + tok0;
@@ -110,6 +222,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     }
                 }
             }
+            if (!ok) break;
+            if (id + NC < total) scalars(id + NC, kidx + 1);
         }
         if (!ok && lane == 0) {
             // gave up: wait (bounded) for the copies still in flight before leaving
@@ -120,90 +234,35 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         }
     } else {
         // ================================ consumer warps ================================================
-        WarpArea &W = S.wa[warp];
         const bool scribe = rank == 0 && warp == 0;     // the one warp that writes the node's record
         int stage = 0;
         uint32_t phase = 0;
         int xn = 0;
+        int kidx = 0;
         float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
 
-        for (long long id = cid; id < total; id += NC) {
+        for (long long id = cid; id < total; id += NC, ++kidx) {
             const int a = (int)(id / P.B), b = (int)(id % P.B);
             const int *parent = P.parent + (long long)b * P.topo_stride;
-            const int *token = P.token + (long long)b * P.N;
             const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
             float s_hi = (float)s_d;
             if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
             float s_lo = (float)(s_d - (double)s_hi);
             if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
 
-            // ---- the node's scalars (the producer's copies are in flight meanwhile) ---------------------------
-            int kc = 0, err = 0;
-            if (lane == 0) {
-                const int pa = __ldg(parent + a);
-                if (a == 0 ? (pa != -1) : (pa < 0 || pa >= a)) err = SPEC_DEV_TOPOLOGY;
-                if (a > 0) {
-                    const int x = __ldg(token + a);
-                    if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
-                }
-            }
-            for (int c0 = a + 1; c0 < P.N; c0 += 32) {
-                const int c = c0 + lane;
-                const bool is = c < P.N && __ldg(parent + c) == a;
-                const unsigned bal = __ballot_sync(0xffffffffu, is);
-                if (is) {
-                    const int pos = kc + __popc(bal & ((1u << lane) - 1u));
-                    if (pos < KMAX) {
-                        const int x = __ldg(token + c);
-                        W.child[pos] = c;
-                        W.cpn[pos] = x;
-                        W.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
-                        if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
-                    }
-                }
-                kc += __popc(bal);
-            }
-            if (kc > KMAX) err = SPEC_DEV_TOPOLOGY;
+            // ---- the node's scalars, gathered by the producer warp --------------------------------------------
+            bool poisoned = *(volatile int *)&S.poison != 0;
+            const NodeScalars &W = S.sc[kidx & 1];
+            if (!poisoned && !mbar_wait(&S.sfull[kidx & 1], (uint32_t)((kidx >> 1) & 1))) { S.poison = 1; poisoned = true; }
+            int err = poisoned ? SPEC_DEV_TIMEOUT : W.err;
+            const int kc = poisoned ? 0 : W.kc;
             const bool hq = kc > 0;
-            // statistics of the node's rows
-            const RowPart *rp = TP.part + ((long long)b * P.N + a) * 2;
-            const double Z_p = __ldcg(&rp[0].S);
-            const int O_p = __ldcg(&rp[0].O);
-            const float cut_p = __ldcg(&rp[0].cut);
-            double Z_q = 0.0;
-            int O_q = ROWPART_EMPTY;
-            float cut_q = -CUDART_INF_F;
-            bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
-            if (hq) {
-                Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
-                bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
-            }
-            err = __reduce_max_sync(0xffffffffu, err);
-            if (bad && !err) err = SPEC_DEV_NONFINITE;
+            const double Z_p = W.Z_p, Z_q = W.Z_q;
+            const int O_p = W.O_p, O_q = W.O_q;
+            const float cut_p = W.cut_p, cut_q = W.cut_q;
             const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
-            // final probabilities of the children's tokens (lanes j: target, 16 + j: draft)
-            __syncwarp();
-            {
-                const int j = lane & 15;
-                const bool mine = !err && j < kc;
-                const int xt = mine ? W.cpn[j] : 0;
-                __syncwarp();
-                if (mine) {
-                    const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
-                    const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + xt);
-                    const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
-                    double pr = 0.0;
-                    if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
-                        const double nd = rint(xd);
-                        pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
-                    }
-                    if (lane < 16) W.cpm[j] = pr; else W.cqm[j] = pr;
-                }
-                __syncwarp();
-            }
 
             // ---- pass 1: e = 2^(z s - O) of both rows, resident ------------------------------------------------
-            bool poisoned = *(volatile int *)&S.poison != 0;
             {
                 const float ofp = (float)O_p, ofq = (float)O_q;
                 RawChunk<DT> raw_p, raw_q;
@@ -389,7 +448,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             // ---- the node's outcome -----------------------------------------------------------------------------
             const double w_fin = (dead || err) ? 0.0 : st_E / st_G;
             bool want_bonus;
-            if (trav) want_bonus = (a == 0) || ((double)__ldg(P.u_accept + (long long)b * P.N + a) < w_fin);
+            if (trav) want_bonus = (a == 0) || ((double)W.u_a < w_fin);
             else want_bonus = acc < 0;
             if (dead || err) want_bonus = false;
             int owner = -1;
@@ -403,7 +462,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             }
             if (want_bonus) {
                 E_tot = warp_sum(lane < C ? E_r : 0.0);
-                const double target = (double)__ldg(P.u_bonus + (long long)b * P.N + a) * E_tot;
+                const double target = (double)W.ub_a * E_tot;
                 owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
             }
             if (scribe) {
@@ -427,80 +486,20 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 split_float(g_commit, gh_c, gl_c);
                 const double invA = 1.0 / A;
                 const double tau_rel = tau * invA, tot_rel = E_tot * invA;       // in units of e
-                for (int i = 0; i < nsm; ++i) {
-                    float p[8], q[8];
-                    const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                    load_e8(d, NCONS, p);
-                    load_e8(d + 2 * NCONS, NCONS, q);
-                    const double r = warp_sum((double)residual_chunk(p, q, gh_c, gl_c));
-                    if (lane == 0) S.wtile[warp][i] = r;
+                const BonusFind bf = bonus_search<NW>(S.wtile, es, nsm, tid, ep0, ep1, ep2, ep3, eq0, eq1, eq2, eq3,
+                                                      gh_c, gl_c, tau_rel);
+                if (bf.role) {
+                    NodeRec &R = P.rec[(long long)b * P.N + a];
+                    R.bonus = bf.role == 1 ? (int)(tok0 + bf.token) : -1;
+                    R.bonus_margin = bf.role == 1 ? (float)(bf.edge / tot_rel) : 0.f;
                 }
-                {
-                    const double r0 = warp_sum((double)residual_chunk(ep0, eq0, gh_c, gl_c));
-                    const double r1 = warp_sum((double)residual_chunk(ep1, eq1, gh_c, gl_c));
-                    const double r2 = warp_sum((double)residual_chunk(ep2, eq2, gh_c, gl_c));
-                    const double r3 = warp_sum((double)residual_chunk(ep3, eq3, gh_c, gl_c));
-                    if (lane == 0) {
-                        S.wtile[warp][nsm] = r0; S.wtile[warp][nsm + 1] = r1;
-                        S.wtile[warp][nsm + 2] = r2; S.wtile[warp][nsm + 3] = r3;
-                    }
-                }
-                bar_sync(1, NCONS);
-                // tile, then warp inside the tile, then lane inside the warp, then token inside the chunk
-                double Ti = 0.0;
-                if (lane < nsm + RT)
-                    for (int w = 0; w < NW; ++w) Ti += S.wtile[w][lane];
-                double tau2, tau3, tau4;
-                const int i_star = pick_lane(Ti, tau_rel, tau2);
-                const double Ww = (i_star >= 0 && lane < NW) ? S.wtile[lane][i_star] : 0.0;
-                const int w_star = i_star >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
-                bar_sync(1, NCONS);          // wtile may be rewritten by the next node only after everyone has read it
-                if (w_star < 0) {
-                    if (warp == 0) {
-                        if (lane == 0) { NodeRec &R = P.rec[(long long)b * P.N + a]; R.bonus = -1; R.bonus_margin = 0.f; }
-                        arrive_sequence(P, b, 1u);
-                    }
-                } else if (warp == w_star) {
-                    float p[8], q[8];
-                    if (i_star < nsm) {
-                        const float4 *d = es + (size_t)(i_star * 4) * NCONS + tid;
-                        load_e8(d, NCONS, p);
-                        load_e8(d + 2 * NCONS, NCONS, q);
-                    } else {
-                        const int jr = i_star - nsm;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
-                            q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
-                        }
-                    }
-                    float wk[8], v = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl_c, q[k], fmaf(-gh_c, q[k], p[k])), 0.f); v += wk[k]; }
-                    const int l_star = pick_lane((double)v, tau3, tau4);
-                    if (lane == l_star) {
-                        double run = 0.0, dlo = 0.0, dhi = 0.0;
-                        int found = -1, last_pos = -1;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const double before = run;
-                            run += (double)wk[k];
-                            if (wk[k] > 0.f) last_pos = k;
-                            if (found < 0 && run > tau4) { found = k; dlo = tau4 - before; dhi = run - tau4; }
-                        }
-                        if (found < 0) { found = last_pos; dlo = 0.0; dhi = 0.0; }
-                        NodeRec &R = P.rec[(long long)b * P.N + a];
-                        R.bonus = found >= 0 ? (int)(tok0 + (long long)i_star * TILE + tid * 8 + found) : -1;
-                        R.bonus_margin = (float)(fmin(dlo, dhi) / tot_rel);
-                    } else if (l_star < 0 && lane == 0) {
-                        NodeRec &R = P.rec[(long long)b * P.N + a];
-                        R.bonus = -1;
-                        R.bonus_margin = 0.f;
-                    }
-                    __syncwarp();
-                    arrive_sequence(P, b, 1u);
-                }
+                // the arrival is made by lane 0 of the warp that holds the reporting thread
+                __syncwarp();
+                if (__any_sync(0xffffffffu, bf.role != 0)) arrive_sequence(P, b, 1u);
             }
+            // the scalars block may be rewritten
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.sempty[kidx & 1]);
         }
     }
     __syncthreads();

@@ -201,6 +201,107 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
     return acc;
 }
 
+// Inverse-CDF search over one CTA's resident residual (e_p - g e_q)+, run by all consumer warps of
+// the CTA that owns the target (tau_rel, in units of e).  Token order is (tile, warp, lane, position
+// in the chunk): the tile, then the warp inside the tile, then the lane, then the token.  The per-tile
+// totals of a warp are reduced together, so that the shuffles of the ten tiles overlap.
+// role: 1 = this thread found the token (index inside the slice in `token`, distance to the nearer
+// CDF edge in `edge`, both in units of e); 2 = this thread reports that no token carries weight;
+// 0 = nothing to do.  wtile is [NW + 1][TMAX] in shared memory; named barrier 1 is used twice.
+struct BonusFind {
+    int role, token;
+    double edge;
+};
+template <int NW>
+__device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const float4 *es, int nsm, int tid,
+                                                  const float (&ep0)[8], const float (&ep1)[8], const float (&ep2)[8],
+                                                  const float (&ep3)[8], const float (&eq0)[8], const float (&eq1)[8],
+                                                  const float (&eq2)[8], const float (&eq3)[8], float gh, float gl,
+                                                  double tau_rel)
+{
+    constexpr int NCONS = NW * 32;
+    constexpr int TILE = NCONS * 8;
+    const int warp = tid >> 5, lane = tid & 31;
+    BonusFind out = {0, -1, 0.0};
+    // slot s < SMT: shared-memory tile s (empty beyond nsm); slot SMT + j: register tile j
+    double r[TMAX];
+#pragma unroll
+    for (int i = 0; i < SMT; ++i) {
+        r[i] = 0.0;
+        if (i < nsm) {
+            float p[8], q[8];
+            const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+            load_e8(d, NCONS, p);
+            load_e8(d + 2 * NCONS, NCONS, q);
+            r[i] = (double)residual_chunk(p, q, gh, gl);
+        }
+    }
+    r[SMT + 0] = (double)residual_chunk(ep0, eq0, gh, gl);
+    r[SMT + 1] = (double)residual_chunk(ep1, eq1, gh, gl);
+    r[SMT + 2] = (double)residual_chunk(ep2, eq2, gh, gl);
+    r[SMT + 3] = (double)residual_chunk(ep3, eq3, gh, gl);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int i = 0; i < TMAX; ++i) r[i] += __shfl_xor_sync(0xffffffffu, r[i], o);
+    }
+#pragma unroll
+    for (int i = 0; i < TMAX; ++i)
+        if (lane == i) wtile[warp][i] = r[i];
+    bar_sync(1, NCONS);
+    double Ti = 0.0;
+    if (lane < TMAX)
+        for (int w = 0; w < NW; ++w) Ti += wtile[w][lane];
+    double tau2, tau3, tau4;
+    const int s_star = pick_lane(Ti, tau_rel, tau2);
+    const double Ww = (s_star >= 0 && lane < NW) ? wtile[lane][s_star] : 0.0;
+    const int w_star = s_star >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
+    bar_sync(1, NCONS);          // wtile may be rewritten only after everyone has read it
+    if (w_star < 0) {
+        if (tid == 0) out.role = 2;
+        return out;
+    }
+    if (warp != w_star) return out;
+    float p[8], q[8];
+    if (s_star < SMT) {
+        const float4 *d = es + (size_t)(s_star * 4) * NCONS + tid;
+        load_e8(d, NCONS, p);
+        load_e8(d + 2 * NCONS, NCONS, q);
+    } else {
+        const int jr = s_star - SMT;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
+            q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
+        }
+    }
+    float wk[8], v = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl, q[k], fmaf(-gh, q[k], p[k])), 0.f); v += wk[k]; }
+    const int l_star = pick_lane((double)v, tau3, tau4);
+    if (l_star < 0) {
+        if (lane == 0) out.role = 2;
+        return out;
+    }
+    if (lane == l_star) {
+        double run = 0.0, dlo = 0.0, dhi = 0.0;
+        int found = -1, last_pos = -1;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const double before = run;
+            run += (double)wk[k];
+            if (wk[k] > 0.f) last_pos = k;
+            if (found < 0 && run > tau4) { found = k; dlo = tau4 - before; dhi = run - tau4; }
+        }
+        if (found < 0) { found = last_pos; dlo = 0.0; dhi = 0.0; }
+        const int tile = s_star < SMT ? s_star : nsm + (s_star - SMT);
+        out.role = found >= 0 ? 1 : 2;
+        out.token = found >= 0 ? tile * TILE + tid * 8 + found : -1;
+        out.edge = fmin(dlo, dhi);
+    }
+    return out;
+}
+
 // Pass 1 for one row of one tile.  The tile's e go to the register array DST (ISREG, a literal) or to
 // shared-memory slot SLOT.  O / SET / SUM / SX / BX: the thread's running reference for this row (an
 // integer-valued float), whether it is set, sum of e, sum of e x and largest exponent.  A chunk whose

@@ -409,73 +409,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 } else if (owner == (int)rank) {
                     float gh_c, gl_c;
                     split_float(g_commit, gh_c, gl_c);
-                    const double tau_rel = tau * rp.Z, tot_rel = E_tot * rp.Z;      // in units of e
-                    for (int i = 0; i < nsm; ++i) {
-                        float p[8], q[8];
-                        const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                        load_e8(d, NCONS, p);
-                        load_e8(d + 2 * NCONS, NCONS, q);
-                        const double r = warp_sum((double)residual_chunk(p, q, gh_c, gl_c));
-                        if (lane == 0) S.wtile[warp][i] = r;
-                    }
-                    {
-                        const double r0 = warp_sum((double)residual_chunk(ep0, eq0, gh_c, gl_c));
-                        const double r1 = warp_sum((double)residual_chunk(ep1, eq1, gh_c, gl_c));
-                        const double r2 = warp_sum((double)residual_chunk(ep2, eq2, gh_c, gl_c));
-                        const double r3 = warp_sum((double)residual_chunk(ep3, eq3, gh_c, gl_c));
-                        if (lane == 0) {
-                            S.wtile[warp][nsm] = r0; S.wtile[warp][nsm + 1] = r1;
-                            S.wtile[warp][nsm + 2] = r2; S.wtile[warp][nsm + 3] = r3;
-                        }
-                    }
-                    bar_sync(1, NCONS);
-                    double Ti = 0.0;
-                    if (lane < nsm + RT)
-                        for (int w = 0; w < NW; ++w) Ti += S.wtile[w][lane];
-                    double tau2, tau3, tau4;
-                    const int i_star = pick_lane(Ti, tau_rel, tau2);
-                    const double Ww = (i_star >= 0 && lane < NW) ? S.wtile[lane][i_star] : 0.0;
-                    const int w_star = i_star >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
-                    bar_sync(1, NCONS);
-                    if (w_star < 0) {
+                    const double tau_rel = tau * rp.Z;      // in units of e
+                    const BonusFind bf = bonus_search<NW>(S.wtile, es, nsm, tid, ep0, ep1, ep2, ep3, eq0, eq1, eq2, eq3,
+                                                          gh_c, gl_c, tau_rel);
+                    if (bf.role == 1) {
+                        bonus = (int)(tok0 + bf.token);
+                        writer = true;
+                    } else if (bf.role == 2) {
                         status = SPEC_DEV_NONFINITE;
-                        if (warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
-                    } else if (warp == w_star) {
-                        float p[8], q[8];
-                        if (i_star < nsm) {
-                            const float4 *d = es + (size_t)(i_star * 4) * NCONS + tid;
-                            load_e8(d, NCONS, p);
-                            load_e8(d + 2 * NCONS, NCONS, q);
-                        } else {
-                            const int jr = i_star - nsm;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
-                                q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
-                            }
-                        }
-                        float wk[8], v = 0.f;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl_c, q[k], fmaf(-gh_c, q[k], p[k])), 0.f); v += wk[k]; }
-                        const int l_star = pick_lane((double)v, tau3, tau4);
-                        if (l_star < 0) {
-                            status = SPEC_DEV_NONFINITE;
-                            if (lane == 0) { writer = true; cur = -1; len = -1; }
-                        } else if (lane == l_star) {
-                            double run = 0.0;
-                            int found = -1, last_pos = -1;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                run += (double)wk[k];
-                                if (wk[k] > 0.f) last_pos = k;
-                                if (found < 0 && run > tau4) found = k;
-                            }
-                            if (found < 0) found = last_pos;
-                            bonus = found >= 0 ? (int)(tok0 + (long long)i_star * TILE + tid * 8 + found) : -1;
-                            writer = true;
-                            if (bonus < 0) { status = SPEC_DEV_NONFINITE; cur = -1; len = -1; }
-                            (void)tot_rel;
-                        }
+                        writer = true; cur = -1; len = -1;
                     }
                 }
             }
