@@ -151,6 +151,16 @@ __device__ __forceinline__ double warp_sum(double v)
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
+// The cluster kernels run long stretches of code once per node or sequence; there the time goes into
+// fetching instructions, not executing them, so their helpers exist once (not inlined) and are warm
+// in the instruction cache after the first call.
+__device__ __noinline__ double warp_sum_once(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __noinline__ double exp2_frac_once(double f) { return exp2_frac(f); }
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll

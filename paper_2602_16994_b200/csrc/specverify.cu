@@ -1,7 +1,9 @@
 // libspecverify: batched draft-tree verification for sm_100a -- host side of the C ABI.
 //
-// Kernels: verify.cuh (the fused SpecInfer / Traversal kernel), rowops.cuh (materialised row
-// distributions, stand-alone inverse CDF), and the residual kernel below.  This file validates
+// Kernels: stream.cuh (row statistics, the one pass over HBM), rowstat.cuh (the same for top-k / top-p
+// rows), walk.cuh (SpecInfer along the accepted path), tree.cuh (every node: Traversal Verification,
+// diagnostic outputs), rowops.cuh (materialised row distributions, stand-alone inverse CDF), and the
+// residual kernel below.  This file validates
 // arguments, chooses the launch plan and enqueues; it never allocates and, except for the
 // host-buffer entry point, never synchronises.
 #include <cuda_runtime.h>
@@ -73,9 +75,9 @@ constexpr int SMEM_2CTA = 113 * 1024;          // so that two CTAs share an SM
 
 inline int up(int x, int m) { return (x + m - 1) / m * m; }
 
-// Smallest cluster whose slices fit on chip: seven consumer warps + the producer warp (256 threads,
-// two CTAs per SM, 128 registers each) while a slice fits in TMAX tiles of 1792 tokens, fifteen
-// consumer warps (one CTA per SM) above that.  SPECVERIFY_CLUSTER / SPECVERIFY_WARPS (environment)
+// Launch shape of the cluster kernels (walk, tree).  Smallest cluster whose slices fit on chip: seven
+// consumer warps + the producer warp (256 threads, two CTAs per SM, 128 registers each) while a slice
+// fits in TMAX tiles of 1792 tokens, fifteen consumer warps (one CTA per SM) above that.  SPECVERIFY_CLUSTER / SPECVERIFY_WARPS (environment)
 // force a cluster size / consumer warp count for tuning.
 bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bool whole_sm = false)
 {
@@ -397,9 +399,9 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
 }
 
 int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl,
-                bool trunc, cudaStream_t st)
+                bool trunc, bool parts, cudaStream_t st)
 {
-    int rc = row_statistics(in, out, w, L, trunc, true, st);
+    int rc = row_statistics(in, out, w, L, trunc, parts, st);
     if (rc) return rc;
     const int NSL = 1;
     RowPart *part = (RowPart *)(w + L.stat);
@@ -416,7 +418,7 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
 }
 
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode,
-                  bool allow_walk = true, bool parts = true)
+                  bool parts = true)
 {
     int rc = check_in(in, true);
     if (rc) return rc;
@@ -430,7 +432,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     cudaStream_t st = (cudaStream_t)stream;
     unsigned char *w = (unsigned char *)ws;
     const bool diagnostics = out->residual || out->node_thr || out->node_w_in || out->margin;
-    if (allow_walk && mode == MODE_SPECINFER && !diagnostics && in->N <= NWALK) {
+    if (mode == MODE_SPECINFER && !diagnostics && in->N <= NWALK) {
         // the walk keeps one cluster per sequence busy: when all of them fit on the chip with one CTA
         // per SM, each CTA may use the whole SM's shared memory for its ring
         VPlan wpl;
@@ -439,7 +441,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
             VPlan big;
             if (make_vplan(in->V, in->logits_dtype, &big, (int)sizeof(WHdr), true) && big.C == wpl.C && big.NW == wpl.NW) wpl = big;
         }
-        return verify_walk(in, out, w, L, wpl, trunc, st);
+        return verify_walk(in, out, w, L, wpl, trunc, parts, st);
     }
     if (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
         cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess) {
@@ -594,7 +596,7 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
     void *ws = nullptr;
     rc = static_ws_address(&ws);
     if (rc) return rc;
-    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false, false);
+    return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false);
 }
 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,

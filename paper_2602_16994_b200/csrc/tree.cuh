@@ -164,7 +164,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
                     if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
                         const double nd = rint(xd);
-                        pr = exp2_frac(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
+                        pr = exp2_frac_once(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
                     }
                 }
                 if (j < KMAX) { if (lane < 16) N.cpm[j] = pr; else N.cqm[j] = pr; }
@@ -283,14 +283,14 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     SPECT_NEXT_TILE(i)
                     float e8[8];
                     unpack_chunk<DT>(raw_p, z);
-                    mask_chunk(z, nvalid, true, cut_p);
+                    mask_chunk(z, nvalid, cut_p > -CUDART_INF_F, cut_p);
                     exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
                     float4 *d = es + (size_t)(i * 4) * NCONS + tid;
                     d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
                     d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
                     if (hq) {
                         unpack_chunk<DT>(raw_q, z);
-                        mask_chunk(z, nvalid, true, cut_q);
+                        mask_chunk(z, nvalid, cut_q > -CUDART_INF_F, cut_q);
                         exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
                         d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
                         d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
@@ -303,11 +303,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 if ((J) < nrg) {                                                                             \
                     SPECT_NEXT_TILE(nsm + (J))                                                               \
                     unpack_chunk<DT>(raw_p, z);                                                              \
-                    mask_chunk(z, nvalid, true, cut_p);                                                      \
+                    mask_chunk(z, nvalid, cut_p > -CUDART_INF_F, cut_p);                                                      \
                     exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                            \
                     if (hq) {                                                                                \
                         unpack_chunk<DT>(raw_q, z);                                                          \
-                        mask_chunk(z, nvalid, true, cut_q);                                                  \
+                        mask_chunk(z, nvalid, cut_q > -CUDART_INF_F, cut_q);                                                  \
                         exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                        \
                     } else {                                                                                 \
                         _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                           \
@@ -366,7 +366,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 }
                 tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
                        (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
-                const double wsum = A * warp_sum((double)tot);
+                const double wsum = A * warp_sum_once((double)tot);
                 const int par = xn & 1;
                 if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
                 if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
@@ -378,7 +378,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
 #pragma unroll
                     for (int w = 0; w < NW; ++w) y += src[w];
                 }
-                return warp_sum(y);
+                return warp_sum_once(y);
             };
 
             bool dead = !(A > 0.0);
@@ -461,7 +461,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 }
             }
             if (want_bonus) {
-                E_tot = warp_sum(lane < C ? E_r : 0.0);
+                E_tot = warp_sum_once(lane < C ? E_r : 0.0);
                 const double target = (double)W.ub_a * E_tot;
                 owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
             }

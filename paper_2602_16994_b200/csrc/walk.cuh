@@ -4,7 +4,7 @@
 // With every row's normaliser known, the decision about a node's FIRST child needs no vocabulary-wide
 // work: its threshold is min(1, p(x)/q(x)), two logits and two normalisers.  The cluster therefore walks
 // down the tree with scalar arithmetic only, and brings a node's rows on chip (the same machinery as
-// the fused kernel: producer warp + bulk-copy ring, e = 2^(z s - O) resident in registers and shared
+// the every-node kernel of tree.cuh: producer warp + bulk-copy ring, e = 2^(z s - O) resident in registers and shared
 // memory, one pass + one distributed-shared-memory exchange per sibling step, inverse-CDF search) only
 // where Algorithm 4 needs a residual: at a node whose first child was rejected, and at the stop node
 // for the bonus draw.  That is one or two resident nodes per sequence instead of every node of the tree.
@@ -216,14 +216,14 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                     const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
                     const float zp_x = load_logit(P.zp, DT, rowb + xt), zq_x = load_logit(P.zq, DT, rowb + xt);
                     double pr[2];
-#pragma unroll
+#pragma unroll 1
                     for (int h = 0; h < 2; ++h) {
                         const float z = h ? zq_x : zp_x;
                         const double xd = (double)z * s_d - (double)S.t_O[2 * a + h];
                         pr[h] = 0.0;
                         if (z >= S.t_cut[2 * a + h] && xd > -1000.0) {
                             const double nd = rint(xd);
-                            pr[h] = exp2_frac(xd - nd) * pow2d((int)nd) * __drcp_rn(S.t_Z[2 * a + h]);
+                            pr[h] = exp2_frac_once(xd - nd) * pow2d((int)nd) * __drcp_rn(S.t_Z[2 * a + h]);
                         }
                     }
                     S.t_cp[c] = pr[0]; S.t_cq[c] = pr[1];
@@ -306,14 +306,14 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                             SPECW_NEXT_TILE(i)
                             float e8[8];
                             unpack_chunk<DT>(raw_p, z);
-                            mask_chunk(z, nvalid, true, rp.cut);
+                            mask_chunk(z, nvalid, rp.cut > -CUDART_INF_F, rp.cut);
                             exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
                             float4 *d = es + (size_t)(i * 4) * NCONS + tid;
                             d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
                             d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
                             if (hq) {
                                 unpack_chunk<DT>(raw_q, z);
-                                mask_chunk(z, nvalid, true, rq.cut);
+                                mask_chunk(z, nvalid, rq.cut > -CUDART_INF_F, rq.cut);
                                 exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
                                 d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
                                 d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
@@ -326,11 +326,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         if ((J) < nrg) {                                                                     \
                             SPECW_NEXT_TILE(nsm + (J))                                                       \
                             unpack_chunk<DT>(raw_p, z);                                                      \
-                            mask_chunk(z, nvalid, true, rp.cut);                                             \
+                            mask_chunk(z, nvalid, rp.cut > -CUDART_INF_F, rp.cut);                                             \
                             exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                    \
                             if (hq) {                                                                        \
                                 unpack_chunk<DT>(raw_q, z);                                                  \
-                                mask_chunk(z, nvalid, true, rq.cut);                                         \
+                                mask_chunk(z, nvalid, rq.cut > -CUDART_INF_F, rq.cut);                                         \
                                 exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                \
                             } else {                                                                         \
                                 _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                   \
@@ -364,7 +364,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         }
                         tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
                                (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
-                        const double wsum = invZp * warp_sum((double)tot);
+                        const double wsum = invZp * warp_sum_once((double)tot);
                         const int par = xn & 1;
                         if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
                         if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
@@ -376,7 +376,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
 #pragma unroll
                             for (int w = 0; w < NW; ++w) y += src[w];
                         }
-                        const double En = warp_sum(y);
+                        const double En = warp_sum_once(y);
                         if (*(volatile int *)&S.poison) { status = SPEC_DEV_TIMEOUT; break; }
                         if (En > 0.0 || j == 0) {
                             if (j > 0) { st_c = cnext; }
@@ -399,7 +399,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
 
                 // ---- stop here: the bonus token from the committed residual ---------------------------------------------
                 done = true;
-                const double E_tot = warp_sum(lane < C ? E_r : 0.0);
+                const double E_tot = warp_sum_once(lane < C ? E_r : 0.0);
                 const double target = (double)S.t_ub[a] * E_tot;
                 double tau;
                 const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);

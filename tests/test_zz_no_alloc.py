@@ -24,7 +24,7 @@ def _outputs_equal(a, b):
 
 
 def test_static_scratch_matches_workspace_entry_point_twice():
-    # the same integer outputs are required bit for bit: both entry points run the same kernel
+    # the same integer outputs are required: decisions of this size sit far from any margin
     shapes = [Workload("na1", 6, 32000, "bf16", 4, 1, 3, 1.0), Workload("na2", 3, 128256, "bf16", 3, 2, 2, 0.8)]
     for call, w in enumerate(shapes):
         batch = make_batch(w, seed=20 + call, device="cuda")
