@@ -38,7 +38,9 @@ struct RParams {
     float T;
     const float *T_seq;
     RowPart *part;             // [B*N*2]: the row's statistics as one slice
-    float *cut;                // [B*N*2] (the verify kernel reads the cuts from here)
+    float *cut;                // [B*N*2] smallest kept logit of every row (for spec_tree_probs)
+    int *todo;                 // [1 + B*N*2]: count, then the ids of the rows the fast path (trunc.cuh) left over
+    int only_todo;             // 1: take only the rows listed in todo
 };
 
 struct __align__(16) Shared {
@@ -245,7 +247,9 @@ __global__ void __launch_bounds__(NT, 2) spec_row_stat_kernel(const RParams P)
 #define SPECV_LEVEL_SHIFT(LV) ((LV) == 0 ? 21 : (DT == SPEC_BF16 ? 16 : ((LV) == 1 ? 10 : 0)))
 #define SPECV_LEVEL_MASK(LV) ((1u << ((LV) == 0 ? 11 : (DT == SPEC_BF16 ? 5 : ((LV) == 1 ? 11 : 10)))) - 1u)
 
-    for (long long id = cid; id < items; id += NC) {
+    const long long n_items = P.only_todo ? (long long)__ldcg(P.todo) : items;
+    for (long long it = cid; it < n_items; it += NC) {
+        const long long id = P.only_todo ? (long long)__ldcg(P.todo + 1 + it) : it;
         const long long row = id >> 1;
         const int which = (int)(id & 1);
         const int b = (int)(row / P.N), a = (int)(row % P.N);

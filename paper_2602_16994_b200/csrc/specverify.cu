@@ -18,6 +18,7 @@
 #include "rowops.cuh"
 #include "rowstat.cuh"
 #include "tree.cuh"
+#include "trunc.cuh"
 #include "specverify.h"
 #include "verify.cuh"
 #include "walk.cuh"
@@ -155,7 +156,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 
 // workspace layout: node records | published weights + arrival counters (cleared per call) | row cuts
 struct WsLayout {
-    int64_t rec, pub, done, cut, stat, clear_bytes, total;
+    int64_t rec, pub, done, cut, todo, stat, clear_bytes, total;
 };
 constexpr int MAX_PARTS = 4;      // parts a row may be split into by the streaming statistics kernel
 WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: one record per row only
@@ -169,6 +170,7 @@ WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: on
     L.clear_bytes = o - L.pub;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
+    L.todo = o; o += up256(4 + nodes * 8);          // count, then ids of the rows left to the general top-k / top-p kernel
     L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // one record per row, then the parts
     L.total = o;
     return L;
@@ -306,9 +308,22 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
     rp.zp = zp; rp.zq = zq; rp.seq_stride = in->seq_stride; rp.node_stride = in->node_stride;
     rp.topo_stride = in->topo_seq_stride; rp.parent = parent; rp.T = in->temperature; rp.T_seq = in->temperature_per_seq;
     rp.part = (RowPart *)(ws + L.stat); rp.cut = (float *)(ws + L.cut);
+    rp.todo = (int *)(ws + L.todo); rp.only_todo = 0;
     const int smem = up(rp.slice_len * esz, 128);
     const long long items = 2ll * in->B * in->N;
     int rc, nc;
+    // fast path first: one CTA per row, selection on a candidate list; the rows it cannot settle are
+    // listed in the workspace and taken by the general kernel afterwards
+    if (cudaMemsetAsync(rp.todo, 0, 4, st) != cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    {
+        const long long want = 2ll * sm_count();
+        const unsigned grid = (unsigned)(items < want ? items : want);
+        if (in->logits_dtype == SPEC_BF16) trunc::spec_row_trunc_kernel<SPEC_BF16><<<grid, trunc::NT, 0, st>>>(rp);
+        else trunc::spec_row_trunc_kernel<SPEC_F32><<<grid, trunc::NT, 0, st>>>(rp);
+        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+        g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
+    }
+    rp.only_todo = 1;
     if (in->logits_dtype == SPEC_BF16) {
         auto k = rowstat::spec_row_stat_kernel<SPEC_BF16>;
         if ((rc = prepare_kernel(k, C, smem))) return rc;
