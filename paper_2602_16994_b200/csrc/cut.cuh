@@ -1,6 +1,7 @@
 // Row cut values for top-k / top-p truncation (the paper's experimental setup names temperature and
 // nucleus sampling; top-k is an addition of the workloads): constants and the key transform; the
-// selection itself runs inside the row-statistics kernel (rowstat.cuh).  The cut of a row is the
+// selection itself runs inside the row-statistics kernels (trunc.cuh: the fast path on candidates;
+// rowstat.cuh: the general kernel for the rows the fast path leaves over).  The cut of a row is the
 // smallest kept logit VALUE:
 //   top-k: the k-th largest logit value (ties at that value are all kept);
 //   top-p: within the top-k set, tokens of equal logit form a group; groups in descending order; the
@@ -9,7 +10,9 @@
 // Both are radix selections on an order-preserving integer image of the logit (sign-flipped bits,
 // -0 folded into +0), 11 bits per level from the top, so equal logits can never be separated and the
 // answer does not depend on token order.  Counts are integers; masses are accumulated as 64-bit fixed
-// point (2^44 per unit of e = exp((z - max)/T)), so every sum is exact and order-free.
+// point (2^44 per unit of e = exp((z - max)/T)), so every sum is exact and order-free.  (One exception:
+// for top-p without top-k the fast path sums the mass of the whole row, which only fixes the target,
+// in floating point to about 1e-7 relative; the masses of the candidates stay exact.)
 #pragma once
 #include "common.cuh"
 

@@ -318,8 +318,14 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
     {
         const long long want = 2ll * sm_count();
         const unsigned grid = (unsigned)(items < want ? items : want);
-        if (in->logits_dtype == SPEC_BF16) trunc::spec_row_trunc_kernel<SPEC_BF16><<<grid, trunc::NT, 0, st>>>(rp);
-        else trunc::spec_row_trunc_kernel<SPEC_F32><<<grid, trunc::NT, 0, st>>>(rp);
+        const bool total = in->top_p < 1.f && !(in->top_k > 0 && in->top_k < in->V);
+        if (in->logits_dtype == SPEC_BF16) {
+            if (total) trunc::spec_row_trunc_kernel<SPEC_BF16, true><<<grid, trunc::NT, 0, st>>>(rp);
+            else trunc::spec_row_trunc_kernel<SPEC_BF16, false><<<grid, trunc::NT, 0, st>>>(rp);
+        } else {
+            if (total) trunc::spec_row_trunc_kernel<SPEC_F32, true><<<grid, trunc::NT, 0, st>>>(rp);
+            else trunc::spec_row_trunc_kernel<SPEC_F32, false><<<grid, trunc::NT, 0, st>>>(rp);
+        }
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
         g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
     }
