@@ -213,15 +213,13 @@ def test_host_buffer_api_matches_device_api():
 TRUNC = [dict(top_k=50), dict(top_p=0.95), dict(top_k=200, top_p=0.9), dict(top_k=1), dict(top_p=0.5)]
 
 
-@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (4099, torch.bfloat16), (128256, torch.bfloat16)])
-@pytest.mark.parametrize("trunc", TRUNC, ids=lambda d: "_".join(f"{k}{v}" for k, v in d.items()))
-def test_tree_probs_truncated(V, dtype, trunc):
+def _check_tree_probs_truncated(V, dtype, trunc, scale=3.0, temperatures=(1.0, 0.6)):
     g = torch.Generator(device="cuda").manual_seed(11)
-    z = (torch.randn((2, 3, V), generator=g, device="cuda") * 3).to(dtype)
+    z = (torch.randn((2, 3, V), generator=g, device="cuda") * scale).to(dtype)
     z[0, 0, : V // 2] = z[0, 0, V // 2: 2 * (V // 2)]          # exact ties everywhere in one row
     z[1, 1, 5] = -0.0
     z[1, 1, 6] = 0.0
-    for T in (1.0, 0.6):
+    for T in temperatures:
         probs, stats = binding.tree_probs(z, 0, temperature=T, **trunc)
         torch.cuda.synchronize()
         zb = z.cpu()
@@ -237,6 +235,23 @@ def test_tree_probs_truncated(V, dtype, trunc):
         assert np.abs(got - rp)[sure].max() < PROB_TOL
         np.testing.assert_array_equal(st[..., 2][sure], rs[..., 2][sure])          # kept count
         np.testing.assert_array_equal(st[..., 5][sure], rs[..., 6][sure].astype(np.float32))   # threshold logit
+
+
+@pytest.mark.parametrize("V,dtype", [(1000, torch.float32), (4099, torch.bfloat16), (128256, torch.bfloat16)])
+@pytest.mark.parametrize("trunc", TRUNC, ids=lambda d: "_".join(f"{k}{v}" for k, v in d.items()))
+def test_tree_probs_truncated(V, dtype, trunc):
+    _check_tree_probs_truncated(V, dtype, trunc)
+
+
+@pytest.mark.parametrize("V,dtype,scale,trunc", [
+    (4099, torch.bfloat16, 0.05, dict(top_p=0.9)),      # flat row: the nucleus window reaches across zero
+    (4099, torch.bfloat16, 3.0, dict(top_k=600)),       # k above what the per-thread maxima can bound
+    (20000, torch.float32, 0.5, dict(top_p=0.9)),       # more candidates than the list holds
+    (20000, torch.float32, 0.5, dict(top_k=3000, top_p=0.99)),
+], ids=["flat_bf16_p", "bf16_k600", "f32_overflow_p", "f32_k3000_p"])
+def test_tree_probs_truncated_rows_left_to_the_general_kernel(V, dtype, scale, trunc):
+    """Rows the candidate-based fast path cannot settle are listed for the general selection kernel."""
+    _check_tree_probs_truncated(V, dtype, trunc, scale=scale, temperatures=(1.0,))
 
 
 TRUNC_SHAPES = [
