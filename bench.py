@@ -32,7 +32,12 @@ ROTATE_BYTES = 4 * L2_BYTES          # bytes touched before an input copy is rea
 # kernels of one call; the roofline figure is taken over the whole call (all of its kernels), so it
 # understates the fraction the streaming kernel reaches on its own
 KERNELS = {"specinfer": "spec_row_partial_kernel + spec_walk_kernel (whole specinfer call)",
-           "traversal": "spec_verify_kernel (whole traversal call)"}
+           "traversal": "spec_row_partial_kernel + spec_tree_kernel (whole traversal call)"}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (cold L2), for the kernels of a SpecInfer call on the headline workload: the row statistics
+# kernel (69.80 + 1.41 MB: every logit once) and the walk kernel (3.96 MB: the rows of the resident
+# nodes, which come from L2 in the benchmark).  Other workloads: not captured.
+TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_800_192 + 1_410_560 + 3_963_136}
 
 
 def parse_args():
@@ -348,7 +353,7 @@ def run_ours(args):
         "per_algorithm": per_algo,
         "roofline": {"bound": "hbm", "kernel": KERNELS[dom], "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                     "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": None,
+                     "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": TRAFFIC_BYTES.get(w.name),
                      "algorithmic_bytes_per_launch": bytes_per_call},
         "clocks": clocks, "gpu_launches": gpu_launches,
         "status_ok": status_ok,

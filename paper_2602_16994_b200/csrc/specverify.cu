@@ -96,7 +96,7 @@ bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bo
             const int slice = up((V + C - 1) / C, 8);
             const int tiles = (slice + tile - 1) / tile;
             if (tiles > TMAX) continue;
-            if (pass == 0 && C > 8) continue;          // prefer one CTA per SM over a non-portable cluster
+            if (pass == 0 && C > 8 && !force_c) continue;   // prefer one CTA per SM over a non-portable cluster
             const int off_x = up(hdr_bytes, 128);
             const int off_es = off_x + up(2 * C * NW * 10 * 8, 128);
             const int es_bytes = (tiles > RT ? tiles - RT : 0) * tile * 8;
@@ -364,12 +364,18 @@ int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
 // start of the statistics region), and the entropy features when asked for.  `parts`: the streaming
 // kernel may split rows into parts (needs the parts region of the workspace).
 int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, bool trunc, bool parts,
-                   cudaStream_t st)
+                   cudaStream_t st, bool init_nodes = false)
 {
     int rc;
     int NSL = 1;
     RowPart *part = (RowPart *)(w + L.stat);
     if (trunc) {
+        if (init_nodes &&
+            (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
+             cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess)) {
+            cudaGetLastError();
+            return SPEC_ERR_CUDA;
+        }
         rc = launch_rowstat(in, in->target_logits, in->draft_logits, in->parent, w, L, st);
         if (rc) return rc;
     } else {
@@ -387,6 +393,7 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
         // in one part is final as written.  One CTA per item: those of unread rows retire at once.
         RowPart *parts = part + 2ll * in->B * in->N;
         sp.part = NSL > 1 ? parts : part;
+        if (init_nodes) { sp.w_pub = (unsigned long long *)(w + L.pub); sp.done = (unsigned int *)(w + L.done); }
         const long long items = 2ll * in->B * in->N * NSL;
         const unsigned grid = (unsigned)(items < (1ll << 20) ? items : (1ll << 20));
         int prc;
@@ -464,13 +471,9 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         }
         return verify_walk(in, out, w, L, wpl, trunc, parts, st);
     }
-    if (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
-        cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess) {
-        cudaGetLastError();
-        return SPEC_ERR_CUDA;
-    }
-    // every node of every sequence on chip once, on top of the row statistics
-    rc = row_statistics(in, out, w, L, trunc, parts, st);
+    // every node of every sequence on chip once, on top of the row statistics (which also set the
+    // published-weight slots to pending and the arrival counters to zero)
+    rc = row_statistics(in, out, w, L, trunc, parts, st, true);
     if (rc) return rc;
     TParams tp = {};
     VParams &vp = tp.v;

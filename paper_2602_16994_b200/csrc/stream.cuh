@@ -37,6 +37,10 @@ struct SParams {
     float T;
     const float *T_seq;
     RowPart *part;           // [B*N*2][NSL]
+    // optional (every-node verification follows): the per-node weight slots are set to pending and the
+    // per-sequence arrival counters to zero here, which saves two memset nodes per call
+    unsigned long long *w_pub;   // [B*N]
+    unsigned int *done;          // [B]
 };
 
 // depth of the per-thread staging ring and its size
@@ -90,6 +94,10 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         const long long row = row2 >> 1;
         const int b = (int)(row / P.N), a = (int)(row % P.N);
         RowPart *out = P.part + row2 * P.NSL + h;
+        if (P.w_pub && which == 0 && h == 0 && tid == 0) {
+            P.w_pub[row] = W_PENDING;
+            if (a == 0) P.done[b] = 0u;
+        }
         if (which == 1) {
             // a draft row is read only for nodes that have children (every warp finds out by itself)
             const int *parent = P.parent + (long long)b * P.topo_stride;
