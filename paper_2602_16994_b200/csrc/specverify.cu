@@ -485,12 +485,10 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
     vp.parent = in->parent; vp.token = in->token;
     vp.T = in->temperature; vp.T_seq = in->temperature_per_seq;
-    vp.cut = nullptr;
     vp.u_accept = in->u_accept; vp.u_bonus = in->u_bonus;
     vp.rec = (NodeRec *)(w + L.rec);
     vp.w_pub = (unsigned long long *)(w + L.pub);
     vp.done = (unsigned int *)(w + L.done);
-    vp.features = nullptr;
     vp.out = *out;
     tp.part = (const RowPart *)(w + L.stat);
     const bool bf = in->logits_dtype == SPEC_BF16;

@@ -52,12 +52,10 @@ struct VParams {
     const int *parent, *token;
     float T;
     const float *T_seq;
-    const float *cut;         // optional [B*N*2]: smallest kept logit of the target / draft row
     const float *u_accept, *u_bonus;
     NodeRec *rec;
     unsigned long long *w_pub;   // [B*N] weight handed to a node by its parent (Traversal), W_PENDING until known
     unsigned int *done;          // [B] arrivals per sequence (two per node); the last one writes the outputs
-    float *features;
     SpecOut out;
 };
 
