@@ -336,7 +336,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         if (bits != W_PENDING || clock64() - t0 > WAIT_CYCLES || *(volatile int *)&S.poison) break;
                         __nanosleep(32);
                     }
-                    __threadfence();
                 }
                 bits = __shfl_sync(0xffffffffu, bits, 0);
                 if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
@@ -391,7 +390,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     if (__ldg(parent + c) == a) {
                         if (trav) {
                             rec[c].w_in = 0.0;
-                            __threadfence();
                             *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
                         } else {
                             rec[c].thr = 0.0;
@@ -409,8 +407,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         NodeRec *rec = P.rec + (long long)b * P.N;
                         const int cj = W.child[j];
                         if (trav) {
+                            // the child polls the published slot only; the record is read after all of the
+                            // sequence's arrivals (each fenced), so no fence is needed between the two stores
                             rec[cj].w_in = thr;
-                            __threadfence();
                             *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
                                 (unsigned long long)__double_as_longlong(thr);
                         } else {
