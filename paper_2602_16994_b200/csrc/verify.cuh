@@ -420,10 +420,11 @@ __device__ __forceinline__ void arrive_sequence(const VParams &P, int b, unsigne
 {
     int last = 0;
     if ((threadIdx.x & 31) == 0) {
-        __threadfence();
-        const unsigned prev = atomicAdd(P.done + b, count);
+        // release: the node's record (written by this warp, ordered before by __syncwarp where another
+        // lane wrote it) is visible to whoever sees the count; acquire: the last arrival sees all records
+        unsigned prev;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(P.done + b), "r"(count) : "memory");
         last = (prev + count == 2u * (unsigned)P.N) ? 1 : 0;
-        if (last) __threadfence();
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) finalize_sequence(P, b);
