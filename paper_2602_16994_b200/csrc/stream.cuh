@@ -63,6 +63,30 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 // asynchronous 16-byte copies (a thread reads back only what it copied itself, so the ring needs no
 // barrier) and keeps a running (reference, sum) pair, rescaled by an exact power of two when a later
 // slice raises its reference.  The CTA reduces once per part.
+// fp32 pairs in one 64-bit register: packed fused multiply-add and add (sm_100)
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
 {
     uint32_t d;
@@ -155,14 +179,21 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
                     if (k & 1) { a1 += e; b1 = fmaf(e, x, b1); } else { a0 += e; b0 = fmaf(e, x, b0); }
                 }
             } else {
-                a0 += ex2_approx(fmaf(z[0], s_lo, fmaf(z[0], s_hi, -of)));
-                a1 += ex2_approx(fmaf(z[1], s_lo, fmaf(z[1], s_hi, -of)));
-                a2 += ex2_approx(fmaf(z[2], s_lo, fmaf(z[2], s_hi, -of)));
-                a3 += ex2_approx(fmaf(z[3], s_lo, fmaf(z[3], s_hi, -of)));
-                a0 += ex2_approx(fmaf(z[4], s_lo, fmaf(z[4], s_hi, -of)));
-                a1 += ex2_approx(fmaf(z[5], s_lo, fmaf(z[5], s_hi, -of)));
-                a2 += ex2_approx(fmaf(z[6], s_lo, fmaf(z[6], s_hi, -of)));
-                a3 += ex2_approx(fmaf(z[7], s_lo, fmaf(z[7], s_hi, -of)));
+                // two logits per instruction: the exponents z s - of and the running sums as fp32 pairs
+                // (each half is the same IEEE operation as the scalar form)
+                const unsigned long long sh2 = pack_f32x2(s_hi, s_hi), sl2 = pack_f32x2(s_lo, s_lo), no2 = pack_f32x2(-of, -of);
+                unsigned long long acc01 = pack_f32x2(a0, a1), acc23 = pack_f32x2(a2, a3);
+#pragma unroll
+                for (int k = 0; k < 8; k += 2) {
+                    const unsigned long long z2 = pack_f32x2(z[k], z[k + 1]);
+                    const unsigned long long x2 = fma_f32x2(z2, sl2, fma_f32x2(z2, sh2, no2));
+                    float x0, x1;
+                    unpack_f32x2(x2, x0, x1);
+                    const unsigned long long e2 = pack_f32x2(ex2_approx(x0), ex2_approx(x1));
+                    if (k & 2) acc23 = add_f32x2(acc23, e2); else acc01 = add_f32x2(acc01, e2);
+                }
+                unpack_f32x2(acc01, a0, a1);
+                unpack_f32x2(acc23, a2, a3);
             }
         };
         auto flush = [&]() {
