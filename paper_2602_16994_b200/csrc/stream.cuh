@@ -63,30 +63,6 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 // asynchronous 16-byte copies (a thread reads back only what it copied itself, so the ring needs no
 // barrier) and keeps a running (reference, sum) pair, rescaled by an exact power of two when a later
 // slice raises its reference.  The CTA reduces once per part.
-// fp32 pairs in one 64-bit register: packed fused multiply-add and add (sm_100)
-__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
-{
-    unsigned long long d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b)
-{
-    unsigned long long d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-
 __device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b)
 {
     uint32_t d;

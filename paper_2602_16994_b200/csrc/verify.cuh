@@ -138,13 +138,26 @@ __device__ __forceinline__ float exp_chunk(const float (&z)[8], float s_hi, floa
                                            float &sx)
 {
     float sum = 0.f;
+    if (FEAT) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        float x = fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of));
-        if (FEAT) x = fmaxf(x, -200.f);
-        e[k] = ex2_approx(x);
-        sum += e[k];
-        if (FEAT) sx = fmaf(e[k], x, sx);
+        for (int k = 0; k < 8; ++k) {
+            const float x = fmaxf(fmaf(z[k], s_lo, fmaf(z[k], s_hi, -of)), -200.f);
+            e[k] = ex2_approx(x);
+            sum += e[k];
+            sx = fmaf(e[k], x, sx);
+        }
+    } else {
+        // two exponents per instruction (fp32 pairs; each half is the scalar operation)
+        const unsigned long long sh2 = pack_f32x2(s_hi, s_hi), sl2 = pack_f32x2(s_lo, s_lo), no2 = pack_f32x2(-of, -of);
+#pragma unroll
+        for (int k = 0; k < 8; k += 2) {
+            const unsigned long long z2 = pack_f32x2(z[k], z[k + 1]);
+            float x0, x1;
+            unpack_f32x2(fma_f32x2(z2, sl2, fma_f32x2(z2, sh2, no2)), x0, x1);
+            e[k] = ex2_approx(x0);
+            e[k + 1] = ex2_approx(x1);
+            sum += e[k] + e[k + 1];
+        }
     }
     return sum;
 }
@@ -179,12 +192,18 @@ __device__ __noinline__ int pick_lane(double v, double tau, double &tau_res)
     return pos ? 31 - __clz(pos) : -1;
 }
 
-// sum over one chunk of (e_p - g e_q)+
+// sum over one chunk of (e_p - g e_q)+, g = gh + gl (two tokens per fused multiply-add)
 __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float (&q)[8], float gh, float gl)
 {
+    const unsigned long long ngh2 = pack_f32x2(-gh, -gh), ngl2 = pack_f32x2(-gl, -gl);
     float acc = 0.f;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) acc += fmaxf(fmaf(-gl, q[k], fmaf(-gh, q[k], p[k])), 0.f);
+    for (int k = 0; k < 8; k += 2) {
+        const unsigned long long q2 = pack_f32x2(q[k], q[k + 1]);
+        float r0, r1;
+        unpack_f32x2(fma_f32x2(ngl2, q2, fma_f32x2(ngh2, q2, pack_f32x2(p[k], p[k + 1]))), r0, r1);
+        acc += fmaxf(r0, 0.f) + fmaxf(r1, 0.f);
+    }
     return acc;
 }
 
