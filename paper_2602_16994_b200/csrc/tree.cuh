@@ -250,6 +250,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             float s_lo = (float)(s_d - (double)s_hi);
             if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
 
+            // Traversal: a first look at the weight the parent may already have published (the load is
+            // in flight while the scalars are waited for).  A weight of exactly 0 means that nothing of this
+            // node can matter (no pass, no exchange, no bonus), so its rows are taken from the ring unread.
+            unsigned long long early = W_PENDING;
+            if (trav && a > 0) early = *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + a);
+
             // ---- the node's scalars, gathered by the producer warp --------------------------------------------
             bool poisoned = *(volatile int *)&S.poison != 0;
             const NodeScalars &W = S.sc[kidx & 1];
@@ -263,7 +269,16 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
 
             // ---- pass 1: e = 2^(z s - O) of both rows, resident ------------------------------------------------
-            {
+            if (__shfl_sync(0xffffffffu, early, 0) == 0ull && !err) {
+                // weight 0: hand the node's stages back without reading them (the decision is per warp; a
+                // node of weight 0 takes part in no exchange, so warps need not agree on it)
+                for (int i = 0; i < ntiles; ++i) {
+                    if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&S.empty[stage]);
+                    if (++stage == NS) { stage = 0; phase ^= 1u; }
+                }
+            } else {
                 const float ofp = (float)O_p, ofq = (float)O_q;
                 RawChunk<DT> raw_p, raw_q;
                 float z[8];
