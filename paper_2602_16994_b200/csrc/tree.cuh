@@ -447,7 +447,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 const double En = pass(g, y);
                 if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
                 if (En > 0.0) {
-                    const double c_new = st_c + st_G, G_new = En + st_G - st_E;
+                    const double c_new = st_c + st_G, G_new = En + (st_G - st_E);   // the difference first: it is exactly 0 while w = 1
                     st_c = c_new; st_G = G_new; st_E = En;
                     g_commit = g;
                     E_r = y;

@@ -312,3 +312,12 @@ def test_cfg3_and_cfg5_sampled():
             assert np.abs(f[..., 0] - sp[..., 3]).max() < 1e-4 and np.abs(f[..., 2] - sp[..., 4]).max() < PROB_TOL
         del full, sub
         torch.cuda.empty_cache()
+
+
+def test_traversal_weight_one_with_a_vanishing_residual():
+    """A node of weight 1 whose residual mass after its child is about 1e-17 (a one-token nucleus that the
+    draft nearly matches): the weight update S / (S + 1 - w) must give 1, not S / ((S + 1) - 1) = S / 0."""
+    w = Workload("t_v1000_f32_p9", 12, 1000, "f32", 2, 1, 3, 1.0, top_p=0.9)
+    batch = make_batch(w, seed=106, device="cuda")
+    check_batch(batch, "traversal", full=True)
+    check_batch(batch, "specinfer", full=True)
