@@ -446,7 +446,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 double y;
                 const double En = pass(g, y);
                 if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
-                if (En > 0.0) {
+                // A residual mass below 1e-10 of the mass before the step is rounding noise of P = q (the e
+                // are fp32): it counts as S = 0, as it is for the exact distributions.
+                if (En > RESIDUAL_FLOOR * st_E) {
                     const double c_new = st_c + st_G, G_new = En + (st_G - st_E);   // the difference first: it is exactly 0 while w = 1
                     st_c = c_new; st_G = G_new; st_E = En;
                     g_commit = g;

@@ -39,6 +39,10 @@ constexpr int NSMAX = 16;    // ring stages
 constexpr int NWMAX = 15;    // consumer warps
 constexpr int OMIN = -(1 << 30);
 constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
+// A residual step whose mass is below this fraction of the mass before it is treated as S = 0: with
+// fp32 exponentials, P = q (for instance two one-token nuclei on the same token) leaves a residual of
+// about 1e-14 instead of exactly nothing.
+constexpr double RESIDUAL_FLOOR = 1.0e-10;
 
 enum Mode { MODE_SPECINFER = 0, MODE_TRAVERSAL = 1 };
 

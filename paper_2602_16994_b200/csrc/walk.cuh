@@ -348,10 +348,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                     // ---- sibling steps (the first child, if any, is already rejected) ------------------------------------
                     const double Rg = hq ? rp.Z * invZq : 0.0;          // pass coefficient g = c Rg (w_in = 1, G = E)
                     int j = j0;
+                    bool have_E = false, redo = false;     // redo: once more with the committed coefficient, for E_r only
                     for (;;) {
                         // one pass + exchange with the coefficient of the current state: c = st_c + (rejections so far)
                         const double cnext = (hq && j > 0) ? st_c + st_E : 0.0;
-                        const double g = cnext * Rg;
+                        const double g = redo ? g_commit : cnext * Rg;
                         float g_hi, g_lo;
                         split_float(g, g_hi, g_lo);
                         float tot = 0.f;
@@ -378,14 +379,21 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         }
                         const double En = warp_sum_once(y);
                         if (*(volatile int *)&S.poison) { status = SPEC_DEV_TIMEOUT; break; }
-                        if (En > 0.0 || j == 0) {
+                        if (redo) { E_r = y; break; }
+                        if (j == 0 || En > RESIDUAL_FLOOR * st_E) {
                             if (j > 0) { st_c = cnext; }
                             st_E = j > 0 ? En : 1.0;
                             g_commit = g;
                             E_r = y;
+                            have_E = true;
                         }
                         // else S = 0 with P equal to q up to rounding: the state stays
-                        if (j >= kc) break;
+                        if (j >= kc) {
+                            // the stop node: if no step was ever committed, the totals of the unchanged P are still missing
+                            if (have_E) break;
+                            redo = true;
+                            continue;
+                        }
                         // child j from the committed state
                         const double Pp = W.cpm[j], Pq = W.cqm[j];
                         const double Ux = Pp - st_c * Pq;
