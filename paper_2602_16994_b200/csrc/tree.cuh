@@ -417,7 +417,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 const double denom = trav ? st_G : st_E;
                 const bool zero = dead || !(Ux > 0.0), one = !zero && !(Pq > 0.0);
                 if (scribe) {
-                    const double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
+                    double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
+                    // Traversal: a weight within 1e-6 of 1 is 1.  With fp32 exponentials a ratio that is exactly
+                    // >= 1 can come out a few 1e-7 below, and the step after it is discontinuous at w = 1 when
+                    // P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
+                    if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
                     if (lane == 0) {
                         NodeRec *rec = P.rec + (long long)b * P.N;
                         const int cj = W.child[j];

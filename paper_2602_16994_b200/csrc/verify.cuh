@@ -43,6 +43,7 @@ constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
 // fp32 exponentials, P = q (for instance two one-token nuclei on the same token) leaves a residual of
 // about 1e-14 instead of exactly nothing.
 constexpr double RESIDUAL_FLOOR = 1.0e-10;
+constexpr double WEIGHT_SNAP = 1.0e-6;      // Traversal: a handed-down weight this close to 1 is 1
 
 enum Mode { MODE_SPECINFER = 0, MODE_TRAVERSAL = 1 };
 
