@@ -35,9 +35,9 @@ KERNELS = {"specinfer": "spec_row_partial_kernel + spec_walk_kernel (whole speci
            "traversal": "spec_row_partial_kernel + spec_tree_kernel (whole traversal call)"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (cold L2), for the kernels of a SpecInfer call on the headline workload: the row statistics
-# kernel (69.80 + 0.86 MB: every logit once) and the walk kernel (4.08 MB: the rows of the resident
+# kernel (69.80 + 0.76 MB: every logit once) and the walk kernel (4.08 MB: the rows of the resident
 # nodes, which come from L2 in the benchmark).  Other workloads: not captured.
-TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_799_168 + 860_672 + 4_075_776}
+TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_798_912 + 760_320 + 4_075_776}
 
 
 def parse_args():
