@@ -10,7 +10,7 @@
 // for the bonus draw.  That is one or two resident nodes per sequence instead of every node of the tree.
 //
 // Before the walk the consumer threads of every CTA bring the sequence's scalars into shared memory in
-// two rounds of independent loads: topology, tokens, uniforms and the row records; then, for every
+// two batches of independent loads: topology, tokens, uniforms and the row records; then, for every
 // non-root node, the two logits at its token in its parent's rows, turned into final probabilities.
 // After that a step down the tree is a few shared-memory reads.
 //
@@ -176,7 +176,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
             float s_lo = (float)(s_d - (double)s_hi);
             if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
 
-            // ---- round 1: topology, tokens, uniforms, row records; the whole tree is checked ----------------------
+            // ---- first batch of loads: topology, tokens, uniforms, row records; the whole tree is checked ---------
             bar_sync(1, NCONS);                      // the previous sequence's scalars are no longer read
             if (tid == 0) S.t_status = 0;
             bar_sync(1, NCONS);
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 if (st1) atomicMax(&S.t_status, st1);
             }
             bar_sync(1, NCONS);
-            // ---- round 2: children, and the probability of every node's token under its parent's rows -------------
+            // ---- second batch of loads: children, and the probability of every node's token under its parent's rows
             if (S.t_status == 0) {
                 int st2 = 0;
                 for (int c = 1 + tid; c < P.N; c += NCONS) {
