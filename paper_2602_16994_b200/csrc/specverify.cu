@@ -8,7 +8,6 @@
 // host-buffer entry point, never synchronises.
 #include <cuda_runtime.h>
 #include <stdint.h>
-#include <stdlib.h>
 
 #include <atomic>
 #include <mutex>
@@ -68,7 +67,7 @@ __global__ void spec_residual_kernel(const RParams P)
 // launch plans
 // ------------------------------------------------------------------------------------------------
 struct VPlan {
-    int C, NW, slice_len, NS, off_x, off_es, off_ring, smem;
+    int C, NW, slice_len, NS, off_x, off_list, off_es, off_ring, smem;
 };
 
 constexpr int SMEM_1CTA = 227 * 1024;          // opt-in limit per CTA
@@ -78,27 +77,24 @@ inline int up(int x, int m) { return (x + m - 1) / m * m; }
 
 // Launch shape of the cluster kernels (walk, tree).  Smallest cluster whose slices fit on chip: seven
 // consumer warps + the producer warp (256 threads, two CTAs per SM, 128 registers each) while a slice
-// fits in TMAX tiles of 1792 tokens, fifteen consumer warps (one CTA per SM) above that.  SPECVERIFY_CLUSTER / SPECVERIFY_WARPS (environment)
-// force a cluster size / consumer warp count for tuning.
+// fits in TMAX tiles of 1792 tokens, fifteen consumer warps (one CTA per SM) above that.
+// Dynamic shared memory: header | exchange slots [2][C][NW][2] doubles | exact lists [NW] | resident e
+// of the tiles that do not fit in registers | ring stages.
 bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bool whole_sm = false)
 {
     const int esz = dtype == SPEC_BF16 ? 2 : 4;
-    int force_c = 0, force_nw = 0;
-    if (const char *e = getenv("SPECVERIFY_CLUSTER")) force_c = atoi(e);
-    if (const char *e = getenv("SPECVERIFY_WARPS")) force_nw = atoi(e);
     for (int pass = 0; pass < 2; ++pass) {
         const int NW = pass == 0 ? 7 : 15;
-        if (force_nw && force_nw != NW) continue;
         const int tile = NW * 32 * 8;
         const int budget = (NW == 7 && !whole_sm) ? SMEM_2CTA : SMEM_1CTA;
         for (int C = 1; C <= CMAX; C <<= 1) {
-            if (force_c && force_c != C) continue;
             const int slice = up((V + C - 1) / C, 8);
             const int tiles = (slice + tile - 1) / tile;
             if (tiles > TMAX) continue;
-            if (pass == 0 && C > 8 && !force_c) continue;   // prefer one CTA per SM over a non-portable cluster
+            if (pass == 0 && C > 8) continue;   // prefer one CTA per SM over a non-portable cluster
             const int off_x = up(hdr_bytes, 128);
-            const int off_es = off_x + up(2 * C * NW * 10 * 8, 128);
+            const int off_list = off_x + up(2 * C * NW * 2 * 8, 128);
+            const int off_es = off_list + up(NW * (int)sizeof(WarpList), 128);
             const int es_bytes = (tiles > RT ? tiles - RT : 0) * tile * 8;
             const int off_ring = off_es + es_bytes;
             const int stage = 2 * tile * esz;
@@ -107,7 +103,8 @@ bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bo
             if (ns > 2 * tiles) ns = 2 * tiles;
             if (ns < 2) continue;
             p->C = C; p->NW = NW; p->slice_len = slice; p->NS = ns;
-            p->off_x = off_x; p->off_es = off_es; p->off_ring = off_ring; p->smem = off_ring + ns * stage;
+            p->off_x = off_x; p->off_list = off_list; p->off_es = off_es; p->off_ring = off_ring;
+            p->smem = off_ring + ns * stage;
             return true;
         }
     }
@@ -435,7 +432,8 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
     RowPart *part = (RowPart *)(w + L.stat);
     WParams wp = {};
     wp.B = in->B; wp.N = in->N; wp.V = in->V; wp.C = pl.C; wp.NSL = NSL;
-    wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.off_x = pl.off_x; wp.off_es = pl.off_es; wp.off_ring = pl.off_ring;
+    wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.off_x = pl.off_x; wp.off_list = pl.off_list; wp.off_es = pl.off_es;
+    wp.off_ring = pl.off_ring;
     wp.zp = in->target_logits; wp.zq = in->draft_logits;
     wp.seq_stride = in->seq_stride; wp.node_stride = in->node_stride; wp.topo_stride = in->topo_seq_stride;
     wp.parent = in->parent; wp.token = in->token; wp.T = in->temperature; wp.T_seq = in->temperature_per_seq;
@@ -480,7 +478,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
     vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
     vp.slice_len = pl.slice_len; vp.NS = pl.NS;
-    vp.off_x = pl.off_x; vp.off_es = pl.off_es; vp.off_ring = pl.off_ring;
+    vp.off_x = pl.off_x; vp.off_list = pl.off_list; vp.off_es = pl.off_es; vp.off_ring = pl.off_ring;
     vp.zp = in->target_logits; vp.zq = in->draft_logits;
     vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
     vp.parent = in->parent; vp.token = in->token;

@@ -4,11 +4,13 @@
 // need (the threshold of every node, Algorithm 4).
 //
 // With a row's reference O and normaliser Z known before the node comes on chip, a node is:
-//   scalars   children, their tokens and uniforms, the final probabilities p(x_c), q(x_c) of every
-//             child's token (two logits and two normalisers each) -- gathered by the producer warp,
-//             one node ahead of the consumers, into a double-buffered block of shared memory;
+//   scalars   children, their tokens and uniforms, the exact exponentials 2^(z s - O) of every child's
+//             token in both rows -- gathered by the producer warp, one node ahead of the consumers,
+//             into a double-buffered block of shared memory;
 //   pass 1    e = 2^(z s - O) of both rows, resident in registers and shared memory, all threads in
-//             the same units (no per-thread references, no exchange of normalisers);
+//             the same units; the dominant tokens in fp64 on the warps' exact lists (verify.cuh);
+//   Z         the rows' normalisers again, from the resident e and the lists (one exchange): the
+//             statistics pass gives them to fp32 accuracy only, too coarse for the differences below;
 //   weight    Traversal: the weight the parent published for this node (bounded poll);
 //   siblings  the residual recursion  U_j = (w_in P0 - c_j q)+,  c_{j+1} = c_j + G_j,
 //             E_j = sum U_j,  G_{j+1} = E_{j+1} + G_j - E_j  (SpecInfer: w_in = 1, G = E), one pass
@@ -32,7 +34,7 @@ struct TParams {
 // what the consumers need to know about a node besides its rows
 struct __align__(16) NodeScalars {
     double Z_p, Z_q;
-    double cpm[KMAX], cqm[KMAX];   // final probabilities of the children's tokens under p and q
+    double cpm[KMAX], cqm[KMAX];   // exact 2^(z s - O) of the children's tokens in the node's target and draft rows
     float cu[KMAX];                // the children's acceptance uniforms
     int child[KMAX];
     int kc, err, O_p, O_q;
@@ -40,7 +42,7 @@ struct __align__(16) NodeScalars {
 };
 
 struct __align__(16) THdr {
-    uint64_t full[NSMAX], empty[NSMAX], xbar[2], sfull[2], sempty[2];
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], cbar, sfull[2], sempty[2];
     double wtile[NWMAX + 1][TMAX];
     NodeScalars sc[2];
     int poison;
@@ -60,7 +62,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     constexpr int STAGE = 2 * ROWB;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     THdr &S = *reinterpret_cast<THdr *>(dyn_smem);
-    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW]
+    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW][2]
+    WarpList *lists = reinterpret_cast<WarpList *>(dyn_smem + P.off_list);   // [warp NW]
     float4 *es = reinterpret_cast<float4 *>(dyn_smem + P.off_es);    // [slot][p lo, p hi, q lo, q hi][NCONS]
     unsigned char *ring = dyn_smem + P.off_ring;
     const int C = P.C, NS = P.NS;
@@ -81,6 +84,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         mbar_init(&S.sfull[1], 1);
         mbar_init(&S.sempty[0], NW);
         mbar_init(&S.sempty[1], NW);
+        mbar_init(&S.cbar, NW);
         S.poison = 0;
         mbar_fence_init();
     }
@@ -150,7 +154,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             }
             err = __reduce_max_sync(0xffffffffu, err);
             if (bad && !err) err = SPEC_DEV_NONFINITE;
-            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
             __syncwarp();
             {
                 const int j = lane & 15;
@@ -164,7 +167,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
                     if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
                         const double nd = rint(xd);
-                        pr = exp2_frac_once(xd - nd) * pow2d((int)nd) * (lane < 16 ? invZp : invZq);
+                        pr = exp2_frac_once(xd - nd) * pow2d((int)nd);
                     }
                 }
                 if (j < KMAX) { if (lane < 16) N.cpm[j] = pr; else N.cqm[j] = pr; }
@@ -235,26 +238,23 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     } else {
         // ================================ consumer warps ================================================
         const bool scribe = rank == 0 && warp == 0;     // the one warp that writes the node's record
+        const RingCtx rc = {S.full, S.empty, ring, NS, &S.poison};
+        WarpList &L = lists[warp];
         int stage = 0;
-        uint32_t phase = 0;
+        uint32_t phase = 0, cph = 0;
         int xn = 0;
         int kidx = 0;
-        float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
+        Resident R;
 
         for (long long id = cid; id < total; id += NC, ++kidx) {
             const int a = (int)(id / P.B), b = (int)(id % P.B);
             const int *parent = P.parent + (long long)b * P.topo_stride;
-            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-            float s_hi = (float)s_d;
-            if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
-            float s_lo = (float)(s_d - (double)s_hi);
-            if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
-
-            // Traversal: a first look at the weight the parent may already have published (the load is
-            // in flight while the scalars are waited for).  A weight of exactly 0 means that nothing of this
-            // node can matter (no pass, no exchange, no bonus), so its rows are taken from the ring unread.
-            unsigned long long early = W_PENDING;
-            if (trav && a > 0) early = *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + a);
+            NodeRows nr;
+            nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+            nr.s_hi = (float)nr.s_d;
+            if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
+            nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
+            if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
 
             // ---- the node's scalars, gathered by the producer warp --------------------------------------------
             bool poisoned = *(volatile int *)&S.poison != 0;
@@ -263,81 +263,28 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             int err = poisoned ? SPEC_DEV_TIMEOUT : W.err;
             const int kc = poisoned ? 0 : W.kc;
             const bool hq = kc > 0;
-            const double Z_p = W.Z_p, Z_q = W.Z_q;
-            const int O_p = W.O_p, O_q = W.O_q;
-            const float cut_p = W.cut_p, cut_q = W.cut_q;
-            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
+            nr.hq = hq; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
+            set_list_thresholds(nr, W.Z_p, W.Z_q);
 
-            // ---- pass 1: e = 2^(z s - O) of both rows, resident ------------------------------------------------
-            if (__shfl_sync(0xffffffffu, early, 0) == 0ull && !err) {
-                // weight 0: hand the node's stages back without reading them (the decision is per warp; a
-                // node of weight 0 takes part in no exchange, so warps need not agree on it)
-                for (int i = 0; i < ntiles; ++i) {
-                    if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&S.empty[stage]);
-                    if (++stage == NS) { stage = 0; phase ^= 1u; }
-                }
-            } else {
-                const float ofp = (float)O_p, ofq = (float)O_q;
-                RawChunk<DT> raw_p, raw_q;
-                float z[8];
-                float dsx = 0.f;
-#define SPECT_NEXT_TILE(TILE_INDEX)                                                                          \
-                if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; }       \
-                {                                                                                            \
-                    const unsigned char *sp_ = ring + (size_t)stage * STAGE + (size_t)tid * 8 * ESZ;         \
-                    raw_p = read_raw<DT>(sp_);                                                               \
-                    if (hq) raw_q = read_raw<DT>(sp_ + ROWB);                                                \
-                }                                                                                            \
-                __syncwarp();                                                                                \
-                if (lane == 0) mbar_arrive(&S.empty[stage]);                                                 \
-                if (++stage == NS) { stage = 0; phase ^= 1u; }                                               \
-                const int nvalid = poisoned ? 0 : n_slice - ((TILE_INDEX) * TILE + tid * 8);
-                for (int i = 0; i < nsm; ++i) {
-                    SPECT_NEXT_TILE(i)
-                    float e8[8];
-                    unpack_chunk<DT>(raw_p, z);
-                    mask_chunk(z, nvalid, cut_p > -CUDART_INF_F, cut_p);
-                    exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
-                    float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                    d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
-                    d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
-                    if (hq) {
-                        unpack_chunk<DT>(raw_q, z);
-                        mask_chunk(z, nvalid, cut_q > -CUDART_INF_F, cut_q);
-                        exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
-                        d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
-                        d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
-                    } else {
-                        d[2 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        d[3 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                }
-#define SPECT_REG_TILE(J, EP, EQ)                                                                            \
-                if ((J) < nrg) {                                                                             \
-                    SPECT_NEXT_TILE(nsm + (J))                                                               \
-                    unpack_chunk<DT>(raw_p, z);                                                              \
-                    mask_chunk(z, nvalid, cut_p > -CUDART_INF_F, cut_p);                                                      \
-                    exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                            \
-                    if (hq) {                                                                                \
-                        unpack_chunk<DT>(raw_q, z);                                                          \
-                        mask_chunk(z, nvalid, cut_q > -CUDART_INF_F, cut_q);                                                  \
-                        exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                        \
-                    } else {                                                                                 \
-                        _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                           \
-                    }                                                                                        \
-                } else {                                                                                     \
-                    _Pragma("unroll") for (int k = 0; k < 8; ++k) { EP[k] = 0.f; EQ[k] = 0.f; }              \
-                }
-                SPECT_REG_TILE(0, ep0, eq0)
-                SPECT_REG_TILE(1, ep1, eq1)
-                SPECT_REG_TILE(2, ep2, eq2)
-                SPECT_REG_TILE(3, ep3, eq3)
-#undef SPECT_REG_TILE
-#undef SPECT_NEXT_TILE
-            }
+            // ---- pass 1: e = 2^(z s - O) of both rows, resident; dominant tokens to the exact lists -------------
+            int nl;
+            float zs_p, zs_q;
+            pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
             if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
+
+            // ---- the rows' normalisers from what is resident (one exchange; a childless node needs none:
+            // its weight is its parent's, and the bonus search works on unnormalised totals) -----------------
+            double Z_p = W.Z_p, Z_q = W.Z_q;
+            if (hq && !err) {
+                const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
+                                     warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
+                double tot[2], mine[2];
+                cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                if (*(volatile int *)&S.poison) err = SPEC_DEV_TIMEOUT;
+                else if (!(tot[0] > 0.0) || !(tot[1] > 0.0)) err = SPEC_DEV_NONFINITE;
+                else { Z_p = tot[0]; Z_q = tot[1]; }
+            }
+            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
 
             // ---- Traversal: the weight handed down by the parent (bounded poll, every warp for itself) ------
             double w_in = 1.0;
@@ -368,31 +315,11 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             // one pass over the resident e with coefficient g, then the exchange: lane r gets rank r's
             // total in y, every lane the cluster's total (bit-identical in every warp of the cluster)
             auto pass = [&](double g, double &y) -> double {
-                float g_hi, g_lo;
-                split_float(g, g_hi, g_lo);
-                float tot = 0.f;
-                for (int i = 0; i < nsm; ++i) {
-                    float p[8], q[8];
-                    const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                    load_e8(d, NCONS, p);
-                    load_e8(d + 2 * NCONS, NCONS, q);
-                    tot += residual_chunk(p, q, g_hi, g_lo);
-                }
-                tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
-                       (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
-                const double wsum = A * warp_sum_once((double)tot);
-                const int par = xn & 1;
-                if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
-                if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
-                if (!*(volatile int *)&S.poison && !mbar_wait_cluster(&S.xbar[par], (uint32_t)((xn >> 1) & 1))) S.poison = 1;
-                ++xn;
-                y = 0.0;
-                if (lane < C) {
-                    const double *src = xchg + (size_t)(par * C + lane) * NW;
-#pragma unroll
-                    for (int w = 0; w < NW; ++w) y += src[w];
-                }
-                return warp_sum_once(y);
+                const double v[1] = {A * warp_sum_once(pass_partial<NW>(es, nsm, tid, R, L, nl, g))};
+                double tot[1], mine[1];
+                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                y = mine[0];
+                return tot[0];
             };
 
             bool dead = !(A > 0.0);
@@ -412,15 +339,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     }
             }
             for (int j = 0; j < kce && !err; ++j) {
-                const double Pp = W.cpm[j], Pq = W.cqm[j];
+                const double Pp = W.cpm[j] * invZp, Pq = W.cqm[j] * invZq;
                 const double Ux = w_in * Pp - st_c * Pq;
                 const double denom = trav ? st_G : st_E;
                 const bool zero = dead || !(Ux > 0.0), one = !zero && !(Pq > 0.0);
                 if (scribe) {
                     double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
-                    // Traversal: a weight within 1e-6 of 1 is 1.  With fp32 exponentials a ratio that is exactly
-                    // >= 1 can come out a few 1e-7 below, and the step after it is discontinuous at w = 1 when
-                    // P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
+                    // Traversal: a weight within 1e-6 of 1 is 1.  The step after it is discontinuous at w = 1
+                    // when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1), and a ratio that is
+                    // exactly >= 1 can come out a rounding below.
                     if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
                     if (lane == 0) {
                         NodeRec *rec = P.rec + (long long)b * P.N;
@@ -450,8 +377,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 double y;
                 const double En = pass(g, y);
                 if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
-                // A residual mass below 1e-10 of the mass before the step is rounding noise of P = q (the e
-                // are fp32): it counts as S = 0, as it is for the exact distributions.
+                // A residual mass below 1e-10 of the mass before the step counts as S = 0 (P equal to q up to
+                // the rounding of the tail's fp32 exponentials), as it is for the exact distributions.
                 if (En > RESIDUAL_FLOOR * st_E) {
                     const double c_new = st_c + st_G, G_new = En + (st_G - st_E);   // the difference first: it is exactly 0 while w = 1
                     st_c = c_new; st_G = G_new; st_E = En;
@@ -487,31 +414,29 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             }
             if (scribe) {
                 if (lane == 0) {
-                    NodeRec &R = P.rec[(long long)b * P.N + a];
-                    R.O_p = (double)O_p; R.Z_p = Z_p; R.O_q = (double)O_q; R.Z_q = Z_q;
-                    R.c_fin = st_c; R.E_fin = (dead || err) ? 0.0 : st_E;
-                    R.cut_p = cut_p; R.cut_q = cut_q;
-                    R.next_child = acc;
-                    R.status = err;
-                    if (trav) { R.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) R.w_in = 1.0; }
-                    else { R.w_in = 1.0; if (a == 0) R.thr = 1.0; }
-                    if (owner < 0) { R.bonus = -1; R.bonus_margin = 0.f; }
+                    NodeRec &Rc = P.rec[(long long)b * P.N + a];
+                    Rc.O_p = (double)nr.O_p; Rc.Z_p = Z_p; Rc.O_q = (double)nr.O_q; Rc.Z_q = Z_q;
+                    Rc.c_fin = st_c; Rc.E_fin = (dead || err) ? 0.0 : st_E;
+                    Rc.cut_p = nr.cut_p; Rc.cut_q = nr.cut_q;
+                    Rc.next_child = acc;
+                    Rc.status = err;
+                    if (trav) { Rc.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) Rc.w_in = 1.0; }
+                    else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
+                    if (owner < 0) { Rc.bonus = -1; Rc.bonus_margin = 0.f; }
                 }
                 arrive_sequence(P, b, owner < 0 ? 2u : 1u);
             }
 
             // ---- bonus token: inverse CDF over the owner CTA's slice -----------------------------------------
             if (owner == (int)rank) {
-                float gh_c, gl_c;
-                split_float(g_commit, gh_c, gl_c);
                 const double invA = 1.0 / A;
                 const double tau_rel = tau * invA, tot_rel = E_tot * invA;       // in units of e
-                const BonusFind bf = bonus_search<NW>(S.wtile, es, nsm, tid, ep0, ep1, ep2, ep3, eq0, eq1, eq2, eq3,
-                                                      gh_c, gl_c, tau_rel);
+                const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl,
+                                                      g_commit, tau_rel);
                 if (bf.role) {
-                    NodeRec &R = P.rec[(long long)b * P.N + a];
-                    R.bonus = bf.role == 1 ? (int)(tok0 + bf.token) : -1;
-                    R.bonus_margin = bf.role == 1 ? (float)(bf.edge / tot_rel) : 0.f;
+                    NodeRec &Rc = P.rec[(long long)b * P.N + a];
+                    Rc.bonus = bf.role == 1 ? (int)(tok0 + bf.token) : (bf.role == 3 ? BONUS_TIMEOUT : -1);
+                    Rc.bonus_margin = bf.role == 1 ? (float)(bf.edge / tot_rel) : 0.f;
                 }
                 // the arrival is made by lane 0 of the warp that holds the reporting thread
                 __syncwarp();

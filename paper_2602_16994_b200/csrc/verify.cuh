@@ -21,6 +21,16 @@
 // over the resident e computing sum (e_p - g e_q)+ plus one scalar exchange through distributed
 // shared memory.
 //
+// Precision.  The e are fp32 (one ex2.approx each, relative error about 2^-22), which is not enough
+// where a residual mass E_j is small against the probabilities it is the difference of (two peaked
+// laws on the same token: near-greedy temperatures, top-k / top-p): w_in P0(x) - c_j q(x) then cancels
+// to a few 1e-7 of its terms.  The few tokens that carry a row's mass are therefore kept exactly: every
+// consumer warp owns a short list of DOMINANT tokens of its part of the slice (above 2^-DOM_A of the
+// row's mass always; above 2^-DOM_B while the list has room), whose exponentials are evaluated in fp64
+// and whose fp32 copies are set to zero.  Every sum over the vocabulary is then (fp32 over the tail,
+// accumulated in fp64 above a thread) + (fp64 over the lists), and so are the rows' normalisers, which
+// the cluster recomputes from the resident e instead of taking them from the statistics pass.
+//
 // Exchanges.  Every consumer warp of every CTA of the cluster sends its partial sum straight into
 // the shared memory of all CTAs (st.async, which counts the bytes on the receiver's mbarrier); every
 // warp waits on its own CTA's mbarrier and reduces all partials itself, in one fixed order, so all
@@ -39,11 +49,18 @@ constexpr int NSMAX = 16;    // ring stages
 constexpr int NWMAX = 15;    // consumer warps
 constexpr int OMIN = -(1 << 30);
 constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
+constexpr int BONUS_TIMEOUT = -2;   // NodeRec::bonus of a node whose bonus search gave up on a wait
 // A residual step whose mass is below this fraction of the mass before it is treated as S = 0: with
 // fp32 exponentials, P = q (for instance two one-token nuclei on the same token) leaves a residual of
 // about 1e-14 instead of exactly nothing.
 constexpr double RESIDUAL_FLOOR = 1.0e-10;
 constexpr double WEIGHT_SNAP = 1.0e-6;      // Traversal: a handed-down weight this close to 1 is 1
+
+// exact list of dominant tokens, one per consumer warp
+constexpr int MW = 32;       // entries (one per lane in a pass)
+constexpr int MW_RES = 8;    // entries kept free for tokens above 2^-DOM_A of a row's mass
+constexpr int DOM_A = 6;     // such a token is always listed: at most 64 per row, and they are what bounds the tail's error
+constexpr int DOM_B = 34;    // tokens above 2^-DOM_B of a row's mass are listed while the list has room
 
 enum Mode { MODE_SPECINFER = 0, MODE_TRAVERSAL = 1 };
 
@@ -51,7 +68,7 @@ struct VParams {
     int B, N, V, C, mode, all_thr;
     int slice_len;            // tokens per CTA slice: a multiple of 8, at most TMAX tiles
     int NS;                   // ring stages
-    int off_x, off_es, off_ring;   // byte offsets inside dynamic shared memory
+    int off_x, off_list, off_es, off_ring;   // byte offsets inside dynamic shared memory
     const void *zp, *zq;
     long long seq_stride, node_stride, topo_stride;
     const int *parent, *token;
@@ -65,8 +82,18 @@ struct VParams {
 };
 
 // per consumer warp: the children of the current node and the scalar state of its recursion
+struct __align__(16) WarpList {
+    double ep[MW], eq[MW];         // exact 2^(z s - O) of the token in the target / draft row (0: cut, or no draft row)
+    int pos[MW];                   // (slot << 8) | (lane << 3) | position in the chunk; slot as in bonus_search
+};
+
+// the e of the RT register tiles of a thread
+struct Resident {
+    float p[RT][8], q[RT][8];
+};
+
 struct __align__(16) WarpArea {
-    double cpm[KMAX], cqm[KMAX];   // final probabilities of the children's tokens under p and q
+    double cpm[KMAX], cqm[KMAX];   // exact 2^(z s - O) of the children's tokens in the node's target and draft rows
     float cu[KMAX];
     int child[KMAX];
     double c, E, G;                // committed state (see the file header); identical in every warp of the cluster
@@ -78,7 +105,7 @@ struct __align__(16) WarpArea {
 };
 
 struct __align__(16) Hdr {
-    uint64_t full[NSMAX], empty[NSMAX], xbar[2];
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], cbar;
     double wtile[NWMAX + 1][TMAX];
     WarpArea wa[NWMAX];
     int poison;
@@ -212,28 +239,273 @@ __device__ __forceinline__ float residual_chunk(const float (&p)[8], const float
     return acc;
 }
 
+// 2^(z s - O) in fp64 (about 1e-15 relative); 0 for -inf and for exponents below the double range
+__device__ __forceinline__ double exp2_exact(float z, double s_d, int O)
+{
+    const double xd = (double)z * s_d - (double)O;
+    if (!(xd > -1000.0)) return 0.0;
+    const double nd = rint(xd);
+    return exp2_frac(xd - nd) * pow2d((int)nd);
+}
+
+// ------------------------------------------------------------------------------------------------
+// pass 1: a node's rows from the ring into resident e, its dominant tokens into the warp's exact list
+// ------------------------------------------------------------------------------------------------
+// what pass 1 has to know about the two rows of a node
+struct NodeRows {
+    bool hq;                  // the node has children: its draft row is read too
+    float cut_p, cut_q;       // smallest kept logit (-inf: nothing cut)
+    int O_p, O_q;             // integer references of the rows
+    float s_hi, s_lo;         // log2(e) / T = s_hi + s_lo
+    double s_d;
+    float thrA_p, thrA_q;     // e above this: always listed (2^-DOM_A of the row's mass)
+    float thrB_p, thrB_q;     // e above this: listed while the list has room (2^-DOM_B)
+};
+// Z: the row's normaliser from the statistics pass (fp32 exponentials: good enough for a threshold)
+__device__ __forceinline__ void set_list_thresholds(NodeRows &nr, double Z_p, double Z_q)
+{
+    nr.thrA_p = (float)(Z_p * (1.0 / (double)(1ull << DOM_A)));
+    nr.thrB_p = (float)(Z_p * (1.0 / (double)(1ull << DOM_B)));
+    nr.thrA_q = nr.hq ? (float)(Z_q * (1.0 / (double)(1ull << DOM_A))) : CUDART_INF_F;
+    nr.thrB_q = nr.hq ? (float)(Z_q * (1.0 / (double)(1ull << DOM_B))) : CUDART_INF_F;
+}
+struct RingCtx {
+    uint64_t *full, *empty;
+    unsigned char *ring;
+    int NS;
+    int *poison;
+};
+
+// Warp-collective: the tokens of this chunk position flagged in m_any (bit k: token k of the lane's
+// chunk; m_a: those above the always-listed threshold) are appended to the warp's list while it has
+// room, their exponentials evaluated in fp64 from the raw logits.  Returns the lane's mask of appended
+// tokens (the caller zeroes their fp32 copies).  n is the list's fill, the same in every lane.
+template <int DT>
+__device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk<DT> raw_p, const RawChunk<DT> raw_q,
+                                             unsigned m_any, unsigned m_a, int nvalid, const NodeRows nr, int slot)
+{
+    const int lane = threadIdx.x & 31;
+    const unsigned lt = (1u << lane) - 1u;
+    float zp[8], zq[8];
+    unpack_chunk<DT>(raw_p, zp);
+    unpack_chunk<DT>(raw_q, zq);
+    unsigned adm = 0;
+#pragma unroll 1
+    for (int k = 0; k < 8; ++k) {
+        const bool a = (m_a >> k) & 1u, b = ((m_any >> k) & 1u) && !a;
+        const unsigned balA = __ballot_sync(0xffffffffu, a), balB = __ballot_sync(0xffffffffu, b);
+        if (!(balA | balB)) continue;
+        const int nA = min(n + __popc(balA), MW);
+        const int capB = MW - MW_RES;
+        const int nB = max(nA, min(nA + __popc(balB), capB));
+        int idx = -1;
+        if (a) { const int i = n + __popc(balA & lt); if (i < MW) idx = i; }
+        else if (b) { const int i = nA + __popc(balB & lt); if (i < capB) idx = i; }
+        n = nB;
+        if (idx >= 0) {
+            float z0 = zp[0], z1 = zq[0];
+#pragma unroll
+            for (int kk = 1; kk < 8; ++kk)
+                if (kk == k) { z0 = zp[kk]; z1 = zq[kk]; }
+            const bool valid = k < nvalid;
+            L.ep[idx] = (valid && z0 >= nr.cut_p) ? exp2_exact(z0, nr.s_d, nr.O_p) : 0.0;
+            L.eq[idx] = (valid && nr.hq && z1 >= nr.cut_q) ? exp2_exact(z1, nr.s_d, nr.O_q) : 0.0;
+            L.pos[idx] = (slot << 8) | (lane << 3) | k;
+            adm |= 1u << k;
+        }
+    }
+    __syncwarp();
+    return adm;
+}
+
+// One tile: wait for the stage, take the thread's 8 logits of both rows, hand the stage back, turn them
+// into e (EP, EQ), move dominant tokens to the list.  The thread's tail sums of e go to zs_p / zs_q.
+template <int DT, int NW>
+__device__ __forceinline__ void pass1_tile(const RingCtx &rc, int &stage, uint32_t &phase, bool &poisoned,
+                                           const NodeRows &nr, int tile_index, int slot, int n_slice, int tid,
+                                           float (&EP)[8], float (&EQ)[8], WarpList &L, int &nl, float &zs_p, float &zs_q)
+{
+    constexpr int NCONS = NW * 32;
+    constexpr int TILE = NCONS * 8;
+    constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
+    constexpr int ROWB = TILE * ESZ;
+    constexpr int STAGE = 2 * ROWB;
+    if (!poisoned && !mbar_wait(&rc.full[stage], phase)) { *rc.poison = 1; poisoned = true; }
+    const unsigned char *sp = rc.ring + (size_t)stage * STAGE + (size_t)tid * 8 * ESZ;
+    const RawChunk<DT> raw_p = read_raw<DT>(sp);
+    RawChunk<DT> raw_q = raw_p;
+    if (nr.hq) raw_q = read_raw<DT>(sp + ROWB);
+    __syncwarp();
+    if ((tid & 31) == 0) mbar_arrive(&rc.empty[stage]);
+    if (++stage == rc.NS) { stage = 0; phase ^= 1u; }
+    const int nvalid = poisoned ? 0 : n_slice - (tile_index * TILE + tid * 8);
+    float z[8], dsx = 0.f;
+    unpack_chunk<DT>(raw_p, z);
+    mask_chunk(z, nvalid, nr.cut_p > -CUDART_INF_F, nr.cut_p);
+    float sum_p = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_p, EP, dsx), sum_q = 0.f;
+    if (nr.hq) {
+        unpack_chunk<DT>(raw_q, z);
+        mask_chunk(z, nvalid, nr.cut_q > -CUDART_INF_F, nr.cut_q);
+        sum_q = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_q, EQ, dsx);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) EQ[k] = 0.f;
+    }
+    // dominant tokens: a chunk whose sum stays below the threshold holds none (e >= 0)
+    const bool room = nl < MW - MW_RES;
+    const float tp = room ? nr.thrB_p : nr.thrA_p, tq = room ? nr.thrB_q : nr.thrA_q;
+    if (__any_sync(0xffffffffu, sum_p > tp || sum_q > tq)) {
+        unsigned m_any = 0, m_a = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const bool a = EP[k] > nr.thrA_p || EQ[k] > nr.thrA_q;
+            const bool any = a || EP[k] > tp || EQ[k] > tq;
+            m_any |= (any ? 1u : 0u) << k;
+            m_a |= (a ? 1u : 0u) << k;
+        }
+        const unsigned adm = list_append<DT>(L, nl, raw_p, raw_q, m_any, m_a, nvalid, nr, slot);
+        if (adm) {
+            sum_p = 0.f; sum_q = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if ((adm >> k) & 1u) { EP[k] = 0.f; EQ[k] = 0.f; }
+                sum_p += EP[k]; sum_q += EQ[k];
+            }
+        }
+    }
+    zs_p += sum_p;
+    zs_q += sum_q;
+}
+
+// Pass 1 of a node.  es: [slot][p lo, p hi, q lo, q hi][NCONS] for the nsm shared-memory tiles; the last
+// nrg tiles of the slice stay in R.  On return nl is the fill of the warp's list and zs_p / zs_q the
+// thread's sums of the fp32 e it keeps (listed tokens excluded).
+template <int DT, int NW>
+__device__ __forceinline__ void pass1(const RingCtx &rc, int &stage, uint32_t &phase, bool &poisoned, const NodeRows &nr,
+                                      float4 *es, int nsm, int nrg, int n_slice, int tid, Resident &R, WarpList &L,
+                                      int &nl, float &zs_p, float &zs_q)
+{
+    constexpr int NCONS = NW * 32;
+    nl = 0; zs_p = 0.f; zs_q = 0.f;
+    for (int i = 0; i < nsm; ++i) {
+        float ep[8], eq[8];
+        pass1_tile<DT, NW>(rc, stage, phase, poisoned, nr, i, i, n_slice, tid, ep, eq, L, nl, zs_p, zs_q);
+        float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+        d[0] = make_float4(ep[0], ep[1], ep[2], ep[3]);
+        d[NCONS] = make_float4(ep[4], ep[5], ep[6], ep[7]);
+        d[2 * NCONS] = make_float4(eq[0], eq[1], eq[2], eq[3]);
+        d[3 * NCONS] = make_float4(eq[4], eq[5], eq[6], eq[7]);
+    }
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+        if (j < nrg) {
+            pass1_tile<DT, NW>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, R.p[j], R.q[j], L, nl, zs_p, zs_q);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { R.p[j][k] = 0.f; R.q[j][k] = 0.f; }
+        }
+    }
+}
+
+// hand a node's stages back unread (the node turned out not to need its rows)
+__device__ __forceinline__ void drain_tiles(const RingCtx &rc, int &stage, uint32_t &phase, bool &poisoned, int ntiles)
+{
+    for (int i = 0; i < ntiles; ++i) {
+        if (!poisoned && !mbar_wait(&rc.full[stage], phase)) { *rc.poison = 1; poisoned = true; }
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(&rc.empty[stage]);
+        if (++stage == rc.NS) { stage = 0; phase ^= 1u; }
+    }
+}
+
+// The thread's share of sum_t (e_p - g e_q)+ over the resident node: its fp32 tail tokens, and the
+// entry of the warp's exact list that falls to its lane.
+template <int NW>
+__device__ __forceinline__ double pass_partial(const float4 *es, int nsm, int tid, const Resident &R, const WarpList &L,
+                                               int nl, double g)
+{
+    constexpr int NCONS = NW * 32;
+    float g_hi, g_lo;
+    split_float(g, g_hi, g_lo);
+    float tot = 0.f;
+    for (int i = 0; i < nsm; ++i) {
+        float p[8], q[8];
+        const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+        load_e8(d, NCONS, p);
+        load_e8(d + 2 * NCONS, NCONS, q);
+        tot += residual_chunk(p, q, g_hi, g_lo);
+    }
+    tot += (residual_chunk(R.p[0], R.q[0], g_hi, g_lo) + residual_chunk(R.p[1], R.q[1], g_hi, g_lo)) +
+           (residual_chunk(R.p[2], R.q[2], g_hi, g_lo) + residual_chunk(R.p[3], R.q[3], g_hi, g_lo));
+    double d = (double)tot;
+    const int lane = tid & 31;
+    if (lane < nl) d += fmax(fma(-g, L.eq[lane], L.ep[lane]), 0.0);
+    return d;
+}
+
+// All-to-all of NV doubles per consumer warp of the cluster: tot[i] is the sum over every warp of every
+// CTA (bit-identical in all of them: one fixed order), mine[i] in lane r < C the sum over CTA r's warps.
+// xchg: [parity 2][rank C][warp NW][2] doubles in every CTA's shared memory, xbar: two mbarriers.
+template <int NW, int NV>
+__device__ __forceinline__ void cluster_exchange(double *xchg, uint64_t *xbar, int &xn, int C, unsigned rank, int warp,
+                                                 int lane, int *poison, const double (&v)[NV], double (&tot)[NV],
+                                                 double (&mine)[NV])
+{
+    static_assert(NV <= 2, "two doubles per warp and exchange at most");
+    const int par = xn & 1;
+    if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&xbar[par], (uint32_t)(C * NW * 8 * NV));
+    if (lane < C) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+            st_async_f64(xchg + ((size_t)(par * C + rank) * NW + warp) * 2 + i, &xbar[par], (uint32_t)lane, v[i]);
+    }
+    if (!*(volatile int *)poison && !mbar_wait_cluster(&xbar[par], (uint32_t)((xn >> 1) & 1))) *poison = 1;
+    ++xn;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) mine[i] = 0.0;
+    if (lane < C) {
+        const double *src = xchg + (size_t)(par * C + lane) * NW * 2;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) mine[i] += src[w * 2 + i];
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) tot[i] = warp_sum_once(mine[i]);
+}
+
+// barrier of the consumer warps of a CTA on an mbarrier (one arrival per warp), with a bounded wait
+__device__ __forceinline__ void consumer_sync(uint64_t *bar, uint32_t &ph, int *poison)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+    if (!*(volatile int *)poison && !mbar_wait(bar, ph)) *poison = 1;
+    ph ^= 1u;
+}
+
 // Inverse-CDF search over one CTA's resident residual (e_p - g e_q)+, run by all consumer warps of
 // the CTA that owns the target (tau_rel, in units of e).  Token order is (tile, warp, lane, position
 // in the chunk): the tile, then the warp inside the tile, then the lane, then the token.  The per-tile
 // totals of a warp are reduced together, so that the shuffles of the ten tiles overlap; warp 0 alone
-// picks tile and warp.
+// picks tile and warp.  Listed tokens enter with their exact values.
 // role: 1 = this thread found the token (index inside the slice in `token`, distance to the nearer
 // CDF edge in `edge`, both in units of e); 2 = this thread reports that no token carries weight;
-// 0 = nothing to do.  wtile is [NW + 1][TMAX] in shared memory; named barrier 1 is used twice.
+// 3 = this thread reports that a bounded wait ran out; 0 = nothing to do.  wtile is [NW + 1][TMAX] in shared memory; cbar / cph: the consumers' barrier.
 struct BonusFind {
     int role, token;
     double edge;
 };
 template <int NW>
-__device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const float4 *es, int nsm, int tid,
-                                                  const float (&ep0)[8], const float (&ep1)[8], const float (&ep2)[8],
-                                                  const float (&ep3)[8], const float (&eq0)[8], const float (&eq1)[8],
-                                                  const float (&eq2)[8], const float (&eq3)[8], float gh, float gl,
-                                                  double tau_rel)
+__device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_t *cbar, uint32_t &cph, int *poison,
+                                                  const float4 *es, int nsm, int tid, const Resident &R,
+                                                  const WarpList &L, int nl, double g, double tau_rel)
 {
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
     const int warp = tid >> 5, lane = tid & 31;
+    float gh, gl;
+    split_float(g, gh, gl);
     BonusFind out = {0, -1, 0.0};
     // slot s < SMT: shared-memory tile s (empty beyond nsm); slot SMT + j: register tile j
     float r[TMAX];
@@ -248,10 +520,8 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const f
             r[i] = residual_chunk(p, q, gh, gl);
         }
     }
-    r[SMT + 0] = residual_chunk(ep0, eq0, gh, gl);
-    r[SMT + 1] = residual_chunk(ep1, eq1, gh, gl);
-    r[SMT + 2] = residual_chunk(ep2, eq2, gh, gl);
-    r[SMT + 3] = residual_chunk(ep3, eq3, gh, gl);
+#pragma unroll
+    for (int j = 0; j < RT; ++j) r[SMT + j] = residual_chunk(R.p[j], R.q[j], gh, gl);
     // a warp's total of one tile: 256 tokens, summed in fp32 like the chunks themselves; every level
     // above works in fp64 on these stored values, so the levels agree with each other exactly
 #pragma unroll
@@ -259,10 +529,22 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const f
 #pragma unroll
         for (int i = 0; i < TMAX; ++i) r[i] += __shfl_xor_sync(0xffffffffu, r[i], o);
     }
+    // the warp's listed tokens, exactly: entry `lane`
+    const double lr = lane < nl ? fmax(fma(-g, L.eq[lane], L.ep[lane]), 0.0) : 0.0;
+    const int lpos = lane < nl ? L.pos[lane] : -1;
+    double mine = 0.0;
 #pragma unroll
     for (int i = 0; i < TMAX; ++i)
-        if (lane == i) wtile[warp][i] = (double)r[i];
-    bar_sync(1, NCONS);
+        if (lane == i) mine = (double)r[i];
+    if (nl > 0) {
+#pragma unroll 1
+        for (int i = 0; i < TMAX; ++i) {
+            const double add = warp_sum_once((lpos >= 0 && (lpos >> 8) == i) ? lr : 0.0);
+            if (lane == i) mine += add;
+        }
+    }
+    if (lane < TMAX) wtile[warp][lane] = mine;
+    consumer_sync(cbar, cph, poison);
     // warp 0 picks the tile and the warp inside it; the others wait for its answer in row NW
     if (warp == 0) {
         double Ti = 0.0;
@@ -274,7 +556,11 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const f
         const int w_pick = s_pick >= 0 ? pick_lane(Ww, tau2, tau3) : -1;
         if (lane == 0) { wtile[NW][0] = (double)s_pick; wtile[NW][1] = (double)w_pick; wtile[NW][2] = tau3; }
     }
-    bar_sync(1, NCONS);
+    consumer_sync(cbar, cph, poison);
+    if (*(volatile int *)poison) {
+        if (tid == 0) out.role = 3;
+        return out;
+    }
     const int s_star = (int)wtile[NW][0], w_star = (int)wtile[NW][1];
     const double tau3 = wtile[NW][2];
     double tau4;
@@ -292,14 +578,27 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const f
         const int jr = s_star - SMT;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            p[k] = jr == 0 ? ep0[k] : (jr == 1 ? ep1[k] : (jr == 2 ? ep2[k] : ep3[k]));
-            q[k] = jr == 0 ? eq0[k] : (jr == 1 ? eq1[k] : (jr == 2 ? eq2[k] : eq3[k]));
+            p[k] = jr == 0 ? R.p[0][k] : (jr == 1 ? R.p[1][k] : (jr == 2 ? R.p[2][k] : R.p[3][k]));
+            q[k] = jr == 0 ? R.q[0][k] : (jr == 1 ? R.q[1][k] : (jr == 2 ? R.q[2][k] : R.q[3][k]));
         }
     }
-    float wk[8], v = 0.f;
+    double wk[8], v = 0.0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) { wk[k] = fmaxf(fmaf(-gl, q[k], fmaf(-gh, q[k], p[k])), 0.f); v += wk[k]; }
-    const int l_star = pick_lane((double)v, tau3, tau4);
+    for (int k = 0; k < 8; ++k) wk[k] = (double)fmaxf(fmaf(-gl, q[k], fmaf(-gh, q[k], p[k])), 0.f);
+    // the listed tokens of this tile: each goes to the lane and position it was taken from
+#pragma unroll 1
+    for (int i = 0; i < nl; ++i) {
+        const int ps = __shfl_sync(0xffffffffu, lpos, i);
+        const double rv = __shfl_sync(0xffffffffu, lr, i);
+        if ((ps >> 8) == s_star && ((ps >> 3) & 31) == lane) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if ((ps & 7) == k) wk[k] = rv;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v += wk[k];
+    const int l_star = pick_lane(v, tau3, tau4);
     if (l_star < 0) {
         if (lane == 0) out.role = 2;
         return out;
@@ -310,8 +609,8 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], const f
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const double before = run;
-            run += (double)wk[k];
-            if (wk[k] > 0.f) last_pos = k;
+            run += wk[k];
+            if (wk[k] > 0.0) last_pos = k;
             if (found < 0 && run > tau4) { found = k; dlo = tau4 - before; dhi = run - tau4; }
         }
         if (found < 0) { found = last_pos; dlo = 0.0; dhi = 0.0; }
@@ -410,7 +709,7 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
         if (acc < 0) status = SPEC_DEV_TOPOLOGY;
     }
     int bonus = acc >= 0 ? __ldcg(&rec[acc].bonus) : -1;
-    if (acc >= 0 && bonus < 0 && !status) status = SPEC_DEV_NONFINITE;
+    if (acc >= 0 && bonus < 0 && !status) status = bonus == BONUS_TIMEOUT ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE;
     if (status) { acc = -1; len = -1; bonus = -1; }
     int *ot = P.out.out_tokens + (long long)b * N;
     for (int i = lane; i < N; i += 32) ot[i] = -1;

@@ -11,8 +11,10 @@
 //
 // Before the walk the consumer threads of every CTA bring the sequence's scalars into shared memory in
 // two batches of independent loads: topology, tokens, uniforms and the row records; then, for every
-// non-root node, the two logits at its token in its parent's rows, turned into final probabilities.
-// After that a step down the tree is a few shared-memory reads.
+// non-root node, the two logits at its token in its parent's rows, exponentiated in fp64.
+// After that a step down the tree is a few shared-memory reads.  The first child's test uses the
+// normalisers of the statistics pass (fp32 exponentials: its threshold is good to a few 1e-7); a node
+// that comes on chip gets its normalisers again from the resident e and the exact lists of verify.cuh.
 //
 // Every consumer warp of the cluster runs the same walk on the same numbers (the exchanges deliver
 // bit-identical totals to all of them), so control flow agrees across the cluster without barriers.
@@ -27,7 +29,7 @@ constexpr int NWALK = 128;        // nodes per sequence the walk keeps in shared
 
 struct WParams {
     int B, N, V, C, NSL;
-    int slice_len, NS, off_x, off_es, off_ring;
+    int slice_len, NS, off_x, off_list, off_es, off_ring;
     const void *zp, *zq;
     long long seq_stride, node_stride, topo_stride;
     const int *parent, *token;
@@ -39,7 +41,7 @@ struct WParams {
 };
 
 struct __align__(16) WHdr {
-    uint64_t full[NSMAX], empty[NSMAX], xbar[2], req, ack;
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], cbar, req, ack;
     double wtile[NWMAX + 1][TMAX];
     WarpArea wa[NWMAX];
     int req_a, req_b, req_hq;
@@ -50,7 +52,7 @@ struct __align__(16) WHdr {
     double t_Z[2 * NWALK];        // normaliser of row (node, target / draft), in units of 2^O
     int t_O[2 * NWALK];
     float t_cut[2 * NWALK];
-    double t_cp[NWALK], t_cq[NWALK];   // probability of the node's token under its parent's p and q
+    double t_cp[NWALK], t_cq[NWALK];   // exact 2^(z s - O) of the node's token in its parent's target and draft rows
     int t_status;
 };
 
@@ -72,7 +74,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
     constexpr int STAGE = 2 * ROWB;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     WHdr &S = *reinterpret_cast<WHdr *>(dyn_smem);
-    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW]
+    double *xchg = reinterpret_cast<double *>(dyn_smem + P.off_x);   // [parity 2][rank C][warp NW][2]
+    WarpList *lists = reinterpret_cast<WarpList *>(dyn_smem + P.off_list);   // [warp NW]
     float4 *es = reinterpret_cast<float4 *>(dyn_smem + P.off_es);    // [slot][p lo, p hi, q lo, q hi][NCONS]
     unsigned char *ring = dyn_smem + P.off_ring;
     const int C = P.C, NS = P.NS;
@@ -89,6 +92,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
         mbar_init(&S.xbar[1], 1);
         mbar_init(&S.req, 1);
         mbar_init(&S.ack, 1);
+        mbar_init(&S.cbar, NW);
         S.poison = 0;
         mbar_fence_init();
     }
@@ -160,21 +164,25 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
     } else {
         // ================================ consumer warps: the walk ==========================================
         WarpArea &W = S.wa[warp];
+        const RingCtx rc = {S.full, S.empty, ring, NS, &S.poison};
+        WarpList &L = lists[warp];
         int stage = 0;
-        uint32_t phase = 0;
+        uint32_t phase = 0, cph = 0;
         int xn = 0;
         uint32_t aphase = 0;        // warp 0, lane 0: requests acknowledged so far (parity)
         bool posted = false;
-        float ep0[8], ep1[8], ep2[8], ep3[8], eq0[8], eq1[8], eq2[8], eq3[8];
+        Resident R;
 
         for (int b = cid; b < P.B; b += NC) {
             const int *parent = P.parent + (long long)b * P.topo_stride;
             const int *token = P.token + (long long)b * P.N;
-            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-            float s_hi = (float)s_d;
-            if ((double)s_hi > s_d) s_hi = __uint_as_float(__float_as_uint(s_hi) - 1u);
-            float s_lo = (float)(s_d - (double)s_hi);
-            if (!(s_lo > 0.f)) s_lo = 1.0e-30f;
+            NodeRows nr;
+            nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+            nr.s_hi = (float)nr.s_d;
+            if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
+            nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
+            if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
+            const double s_d = nr.s_d;
 
             // ---- first batch of loads: topology, tokens, uniforms, row records; the whole tree is checked ---------
             bar_sync(1, NCONS);                      // the previous sequence's scalars are no longer read
@@ -206,7 +214,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 if (st1) atomicMax(&S.t_status, st1);
             }
             bar_sync(1, NCONS);
-            // ---- second batch of loads: children, and the probability of every node's token under its parent's rows
+            // ---- second batch of loads: children, and the exponential of every node's token in its parent's rows
             if (S.t_status == 0) {
                 int st2 = 0;
                 for (int c = 1 + tid; c < P.N; c += NCONS) {
@@ -223,7 +231,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         pr[h] = 0.0;
                         if (z >= S.t_cut[2 * a + h] && xd > -1000.0) {
                             const double nd = rint(xd);
-                            pr[h] = exp2_frac_once(xd - nd) * pow2d((int)nd) * __drcp_rn(S.t_Z[2 * a + h]);
+                            pr[h] = exp2_frac_once(xd - nd) * pow2d((int)nd);
                         }
                     }
                     S.t_cp[c] = pr[0]; S.t_cq[c] = pr[1];
@@ -247,7 +255,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 rp.Z = S.t_Z[2 * a]; rp.O = S.t_O[2 * a]; rp.cut = S.t_cut[2 * a];
                 rq = rp;
                 if (hq) { rq.Z = S.t_Z[2 * a + 1]; rq.O = S.t_O[2 * a + 1]; rq.cut = S.t_cut[2 * a + 1]; }
-                const double invZp = __drcp_rn(rp.Z), invZq = hq ? __drcp_rn(rq.Z) : 0.0;
                 // ---- first child: needs no residual -------------------------------------------------------------------
                 bool resident = false;
                 double st_c = 0.0, st_E = 1.0, g_commit = 0.0;
@@ -255,9 +262,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 int acc = -1;
                 int j0 = 0;
                 if (hq) {
-                    const double Pp = S.t_cp[c_first], Pq = S.t_cq[c_first];
-                    const bool zero = !(Pp > 0.0), one = !zero && !(Pq > 0.0);
-                    if (!zero && (one || (double)S.t_u[c_first] * Pq < Pp)) acc = c_first;
+                    // p(x) / q(x) = (e_p / Z_p) / (e_q / Z_q), written without a division
+                    const double ep = S.t_cp[c_first], eq = S.t_cq[c_first];
+                    const bool zero = !(ep > 0.0), one = !zero && !(eq > 0.0);
+                    if (!zero && (one || (double)S.t_u[c_first] * eq * rp.Z < ep * rq.Z)) acc = c_first;
                     j0 = 1;
                 }
                 if (acc < 0) {
@@ -286,98 +294,33 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         posted = true;
                     }
                     bool poisoned = *(volatile int *)&S.poison != 0;
-                    const float ofp = (float)rp.O, ofq = (float)rq.O;
-                    {
-                        RawChunk<DT> raw_p, raw_q;
-                        float z[8];
-                        float dsx = 0.f;
-#define SPECW_NEXT_TILE(TILE_INDEX)                                                                          \
-                        if (!poisoned && !mbar_wait(&S.full[stage], phase)) { S.poison = 1; poisoned = true; } \
-                        {                                                                                    \
-                            const unsigned char *sp_ = ring + (size_t)stage * STAGE + (size_t)tid * 8 * ESZ; \
-                            raw_p = read_raw<DT>(sp_);                                                       \
-                            if (hq) raw_q = read_raw<DT>(sp_ + ROWB);                                        \
-                        }                                                                                    \
-                        __syncwarp();                                                                        \
-                        if (lane == 0) mbar_arrive(&S.empty[stage]);                                         \
-                        if (++stage == NS) { stage = 0; phase ^= 1u; }                                       \
-                        const int nvalid = poisoned ? 0 : n_slice - ((TILE_INDEX) * TILE + tid * 8);
-                        for (int i = 0; i < nsm; ++i) {
-                            SPECW_NEXT_TILE(i)
-                            float e8[8];
-                            unpack_chunk<DT>(raw_p, z);
-                            mask_chunk(z, nvalid, rp.cut > -CUDART_INF_F, rp.cut);
-                            exp_chunk<FEAT>(z, s_hi, s_lo, ofp, e8, dsx);
-                            float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                            d[0] = make_float4(e8[0], e8[1], e8[2], e8[3]);
-                            d[NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
-                            if (hq) {
-                                unpack_chunk<DT>(raw_q, z);
-                                mask_chunk(z, nvalid, rq.cut > -CUDART_INF_F, rq.cut);
-                                exp_chunk<FEAT>(z, s_hi, s_lo, ofq, e8, dsx);
-                                d[2 * NCONS] = make_float4(e8[0], e8[1], e8[2], e8[3]);
-                                d[3 * NCONS] = make_float4(e8[4], e8[5], e8[6], e8[7]);
-                            } else {
-                                d[2 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                d[3 * NCONS] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            }
-                        }
-#define SPECW_REG_TILE(J, EP, EQ)                                                                            \
-                        if ((J) < nrg) {                                                                     \
-                            SPECW_NEXT_TILE(nsm + (J))                                                       \
-                            unpack_chunk<DT>(raw_p, z);                                                      \
-                            mask_chunk(z, nvalid, rp.cut > -CUDART_INF_F, rp.cut);                                             \
-                            exp_chunk<FEAT>(z, s_hi, s_lo, ofp, EP, dsx);                                    \
-                            if (hq) {                                                                        \
-                                unpack_chunk<DT>(raw_q, z);                                                  \
-                                mask_chunk(z, nvalid, rq.cut > -CUDART_INF_F, rq.cut);                                         \
-                                exp_chunk<FEAT>(z, s_hi, s_lo, ofq, EQ, dsx);                                \
-                            } else {                                                                         \
-                                _Pragma("unroll") for (int k = 0; k < 8; ++k) EQ[k] = 0.f;                   \
-                            }                                                                                \
-                        } else {                                                                             \
-                            _Pragma("unroll") for (int k = 0; k < 8; ++k) { EP[k] = 0.f; EQ[k] = 0.f; }      \
-                        }
-                        SPECW_REG_TILE(0, ep0, eq0)
-                        SPECW_REG_TILE(1, ep1, eq1)
-                        SPECW_REG_TILE(2, ep2, eq2)
-                        SPECW_REG_TILE(3, ep3, eq3)
-#undef SPECW_REG_TILE
-#undef SPECW_NEXT_TILE
+                    nr.hq = hq; nr.cut_p = rp.cut; nr.cut_q = rq.cut; nr.O_p = rp.O; nr.O_q = rq.O;
+                    set_list_thresholds(nr, rp.Z, rq.Z);
+                    int nl;
+                    float zs_p, zs_q;
+                    pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
+                    // ---- the rows' normalisers from what is resident (needed only where a sibling step follows)
+                    double Z_p = rp.Z, Z_q = rq.Z;
+                    if (hq) {
+                        const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
+                                             warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
+                        double tot[2], mine[2];
+                        cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                        if (tot[0] > 0.0 && tot[1] > 0.0) { Z_p = tot[0]; Z_q = tot[1]; }
                     }
+                    const double invZp = __drcp_rn(Z_p), invZq = hq ? __drcp_rn(Z_q) : 0.0;
                     // ---- sibling steps (the first child, if any, is already rejected) ------------------------------------
-                    const double Rg = hq ? rp.Z * invZq : 0.0;          // pass coefficient g = c Rg (w_in = 1, G = E)
+                    const double Rg = hq ? Z_p * invZq : 0.0;          // pass coefficient g = c Rg (w_in = 1, G = E)
                     int j = j0;
                     bool have_E = false, redo = false;     // redo: once more with the committed coefficient, for E_r only
                     for (;;) {
                         // one pass + exchange with the coefficient of the current state: c = st_c + (rejections so far)
                         const double cnext = (hq && j > 0) ? st_c + st_E : 0.0;
                         const double g = redo ? g_commit : cnext * Rg;
-                        float g_hi, g_lo;
-                        split_float(g, g_hi, g_lo);
-                        float tot = 0.f;
-                        for (int i = 0; i < nsm; ++i) {
-                            float p[8], q[8];
-                            const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-                            load_e8(d, NCONS, p);
-                            load_e8(d + 2 * NCONS, NCONS, q);
-                            tot += residual_chunk(p, q, g_hi, g_lo);
-                        }
-                        tot += (residual_chunk(ep0, eq0, g_hi, g_lo) + residual_chunk(ep1, eq1, g_hi, g_lo)) +
-                               (residual_chunk(ep2, eq2, g_hi, g_lo) + residual_chunk(ep3, eq3, g_hi, g_lo));
-                        const double wsum = invZp * warp_sum_once((double)tot);
-                        const int par = xn & 1;
-                        if (warp == 0 && lane == 0) mbar_arrive_expect_tx(&S.xbar[par], (uint32_t)(C * NW * 8));
-                        if (lane < C) st_async_f64(xchg + (size_t)(par * C + rank) * NW + warp, &S.xbar[par], (uint32_t)lane, wsum);
-                        if (!*(volatile int *)&S.poison && !mbar_wait_cluster(&S.xbar[par], (uint32_t)((xn >> 1) & 1))) S.poison = 1;
-                        ++xn;
-                        double y = 0.0;
-                        if (lane < C) {
-                            const double *src = xchg + (size_t)(par * C + lane) * NW;
-#pragma unroll
-                            for (int w = 0; w < NW; ++w) y += src[w];
-                        }
-                        const double En = warp_sum_once(y);
+                        const double v[1] = {invZp * warp_sum_once(pass_partial<NW>(es, nsm, tid, R, L, nl, g))};
+                        double tot[1], mine[1];
+                        cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                        const double En = tot[0], y = mine[0];
                         if (*(volatile int *)&S.poison) { status = SPEC_DEV_TIMEOUT; break; }
                         if (redo) { E_r = y; break; }
                         if (j == 0 || En > RESIDUAL_FLOOR * st_E) {
@@ -395,39 +338,39 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                             continue;
                         }
                         // child j from the committed state
-                        const double Pp = W.cpm[j], Pq = W.cqm[j];
+                        const double Pp = W.cpm[j] * invZp, Pq = W.cqm[j] * invZq;
                         const double Ux = Pp - st_c * Pq;
                         const bool zero = !(Ux > 0.0), one = !zero && !(Pq > 0.0);
                         if (!zero && (one || (double)W.cu[j] * st_E * Pq < Ux)) { acc = W.child[j]; break; }
                         ++j;
                     }
                     if (status) { done = true; if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; } break; }
-                }
-                if (acc >= 0) { cur = acc; ++len; continue; }
-
-                // ---- stop here: the bonus token from the committed residual ---------------------------------------------
-                done = true;
-                const double E_tot = warp_sum_once(lane < C ? E_r : 0.0);
-                const double target = (double)S.t_ub[a] * E_tot;
-                double tau;
-                const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
-                if (owner < 0) {
-                    status = SPEC_DEV_NONFINITE;
-                    if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
-                } else if (owner == (int)rank) {
-                    float gh_c, gl_c;
-                    split_float(g_commit, gh_c, gl_c);
-                    const double tau_rel = tau * rp.Z;      // in units of e
-                    const BonusFind bf = bonus_search<NW>(S.wtile, es, nsm, tid, ep0, ep1, ep2, ep3, eq0, eq1, eq2, eq3,
-                                                          gh_c, gl_c, tau_rel);
-                    if (bf.role == 1) {
-                        bonus = (int)(tok0 + bf.token);
-                        writer = true;
-                    } else if (bf.role == 2) {
-                        status = SPEC_DEV_NONFINITE;
-                        writer = true; cur = -1; len = -1;
+                    if (acc < 0) {
+                        // ---- stop here: the bonus token from the committed residual ---------------------------------------
+                        done = true;
+                        const double E_tot = warp_sum_once(lane < C ? E_r : 0.0);
+                        const double target = (double)S.t_ub[a] * E_tot;
+                        double tau;
+                        const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
+                        if (owner < 0) {
+                            status = SPEC_DEV_NONFINITE;
+                            if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
+                        } else if (owner == (int)rank) {
+                            const double tau_rel = tau * Z_p;      // in units of e
+                            const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl,
+                                                                  g_commit, tau_rel);
+                            if (bf.role == 1) {
+                                bonus = (int)(tok0 + bf.token);
+                                writer = true;
+                            } else if (bf.role >= 2) {
+                                status = bf.role == 3 ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE;
+                                writer = true; cur = -1; len = -1;
+                            }
+                        }
                     }
                 }
+                (void)resident;
+                if (acc >= 0) { cur = acc; ++len; continue; }
             }
 
             // ---- outputs of the sequence (one thread) -----------------------------------------------------------------------

@@ -4,12 +4,8 @@ batch and compare them under the stated rules.
 Rules.  Integer outputs (accepted node, path tokens, bonus token) must be identical, except where
 the oracle itself says the decision was closer than 1e-6 to its threshold (|u - thr| for an
 acceptance test, distance to the CDF boundary as a fraction of the total mass for the bonus draw);
-such differences are counted and reported, anything else fails.  Probabilities, residuals and
-weights must agree within 1e-5 absolute.  The per-node thresholds reported for diagnosis divide by
-the residual mass E = sum (P - c q)+, which the device forms from fp32 exponentials (relative error
-about 2^-22 each): where a peaked P and q nearly coincide, E is a small difference of large terms
-and the threshold inherits a relative error of about 2^-22 (max P + c max q) / E.  They must agree
-within 1e-5 on all but 2 % of the nodes (at least one node is allowed) and within 1e-4 everywhere.
+such differences are counted and reported, anything else fails.  Probabilities, residuals, per-node
+thresholds, weights and margins must agree within 1e-5 absolute, every entry.
 """
 from __future__ import annotations
 
@@ -24,13 +20,11 @@ from paper_2602_16994_b200 import binding
 
 MARGIN = 1e-6
 PROB_TOL = 1e-5
-THR_TOL_WORST = 1e-4
 
 
 def assert_thresholds(got, ref, what):
     d = np.abs(np.asarray(got, np.float64) - ref)
-    assert d.max(initial=0.0) < THR_TOL_WORST, f"{what} differ by {d.max():.3e}"
-    assert (d >= PROB_TOL).sum() <= max(1, int(0.02 * d.size)), f"{what}: {(d >= PROB_TOL).sum()} of {d.size} nodes differ by more than 1e-5"
+    assert d.max(initial=0.0) < PROB_TOL, f"{what} differ by {d.max():.3e}"
 
 
 def oracle_inputs(batch) -> TreeInputs:
@@ -140,5 +134,5 @@ def check_batch(batch, algo, full=True) -> Tally:
     mg = got.margin.cpu().numpy()
     ua = inp.u_accept.astype(np.float64)
     ref_thr = ratio if algo == "specinfer" else w_fin
-    assert np.abs(mg[:, 1:N] - np.abs(ua[:, 1:] - ref_thr[:, 1:])).max(initial=0.0) < THR_TOL_WORST
+    assert np.abs(mg[:, 1:N] - np.abs(ua[:, 1:] - ref_thr[:, 1:])).max(initial=0.0) < PROB_TOL
     return tally
