@@ -416,7 +416,10 @@ static int trav_visit(Trav *tv, int a, double w)
                 double d = w * P[t] - Q[t];
                 P[t] = d > 0.0 ? d / S : 0.0;
             }
-            w = S / (S + 1.0 - w);
+            /* the sum is formed as S + (1 - w): 1 - w is exact for w in [1/2, 1], so a weight of exactly 1
+             * stays exactly 1; (S + 1) - w would round S to the grid of 1 and the deviation of w from 1
+             * grows by 1/S with every later step */
+            w = S / (S + (1.0 - w));
         } else {
             w = (w >= 1.0) ? 1.0 : 0.0;
         }

@@ -307,7 +307,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             // ---- state of the recursion (identical in every warp of the cluster) ------------------------------
             const bool live = !err && w_in > 0.0;
             const double A = live ? w_in * invZp : 0.0;
-            const double Rg = (live && hq) ? Z_p * invZq * (w_in == 1.0 ? 1.0 : __drcp_rn(w_in)) : 0.0;
+            // a true division: equal normalisers and w_in = 1 give exactly 1
+            const double Rg = (live && hq) ? __ddiv_rn(Z_p, w_in == 1.0 ? Z_q : w_in * Z_q) : 0.0;
             double st_c = 0.0, st_E = err ? 0.0 : w_in, st_G = 1.0, g_commit = 0.0;
             double E_r = 0.0;            // lane r: rank r's total of the committed U
             bool have_E = false;
@@ -345,9 +346,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 const bool zero = dead || !(Ux > 0.0), one = !zero && !(Pq > 0.0);
                 if (scribe) {
                     double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
-                    // Traversal: a weight within 1e-6 of 1 is 1.  The step after it is discontinuous at w = 1
-                    // when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1), and a ratio that is
-                    // exactly >= 1 can come out a rounding below.
+                    // Traversal: a weight within a rounding of 1 is 1.  The step after it is discontinuous at
+                    // w = 1 when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
                     if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
                     if (lane == 0) {
                         NodeRec *rec = P.rec + (long long)b * P.N;

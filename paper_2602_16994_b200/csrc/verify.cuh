@@ -50,11 +50,13 @@ constexpr int NWMAX = 15;    // consumer warps
 constexpr int OMIN = -(1 << 30);
 constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
 constexpr int BONUS_TIMEOUT = -2;   // NodeRec::bonus of a node whose bonus search gave up on a wait
-// A residual step whose mass is below this fraction of the mass before it is treated as S = 0: with
-// fp32 exponentials, P = q (for instance two one-token nuclei on the same token) leaves a residual of
-// about 1e-14 instead of exactly nothing.
-constexpr double RESIDUAL_FLOOR = 1.0e-10;
-constexpr double WEIGHT_SNAP = 1.0e-6;      // Traversal: a handed-down weight this close to 1 is 1
+// A residual step whose mass is below this fraction of the mass before it is treated as S = 0: where P
+// equals q (the same row twice, two one-token nuclei on the same token) the exact difference is 0 and
+// the computed one a few 1e-16 of the mass (the rounding of the coefficient g).
+constexpr double RESIDUAL_FLOOR = 1.0e-13;
+// Traversal: a handed-down weight this close to 1 is 1 (a ratio that is exactly 1 may come out one
+// rounding below; the step after it is discontinuous at w = 1 when S = 0)
+constexpr double WEIGHT_SNAP = 1.0e-12;
 
 // exact list of dominant tokens, one per consumer warp
 constexpr int MW = 32;       // entries (one per lane in a pass)

@@ -310,7 +310,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                     }
                     const double invZp = __drcp_rn(Z_p), invZq = hq ? __drcp_rn(Z_q) : 0.0;
                     // ---- sibling steps (the first child, if any, is already rejected) ------------------------------------
-                    const double Rg = hq ? Z_p * invZq : 0.0;          // pass coefficient g = c Rg (w_in = 1, G = E)
+                    const double Rg = hq ? __ddiv_rn(Z_p, Z_q) : 0.0;   // pass coefficient g = c Rg (w_in = 1, G = E); equal normalisers give exactly 1
                     int j = j0;
                     bool have_E = false, redo = false;     // redo: once more with the committed coefficient, for E_r only
                     for (;;) {

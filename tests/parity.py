@@ -48,11 +48,46 @@ class Tally:
     decisions: int = 0
     near_margin_mismatches: int = 0
     near_margin_decisions: int = 0
+    sequences: int = 0
+    rows: int = 0                 # logit rows whose cut (top-k / top-p) was compared
+    rows_near_boundary: int = 0   # of those: nucleus boundary within 1e-6 of top_p (the oracle's own margin)
+    rows_cut_differs: int = 0     # of those: the device kept a different set (tolerated only near the boundary)
+    sequences_set_aside: int = 0  # sequences holding such a row: their outputs are not compared
 
     def add(self, other):
-        self.decisions += other.decisions
-        self.near_margin_mismatches += other.near_margin_mismatches
-        self.near_margin_decisions += other.near_margin_decisions
+        for k in vars(self):
+            setattr(self, k, getattr(self, k) + getattr(other, k))
+
+
+def settle_cuts(batch, inp, tally: Tally):
+    """Truncating workloads: compare the cut (smallest kept logit) the device chose for every row the
+    verifiers read with the oracle's.  A different cut is tolerated only where the oracle says the
+    nucleus boundary lies within 1e-6 of top_p; the sequences that hold such a row are returned (their
+    distributions legitimately differ there) and counted."""
+    w = batch.workload
+    B, N, V = inp.shape
+    parent = batch.parent.cpu().numpy()
+    internal = np.zeros(N, bool); internal[parent[1:]] = True
+    bad_seq = np.zeros(B, bool)
+    for which, rows in ((0, np.ones(N, bool)), (1, internal)):
+        logits = batch.target_logits if which == 0 else batch.draft_logits
+        _, st = binding.tree_probs(logits, 0, temperature=w.temperature, top_k=w.top_k, top_p=w.top_p,
+                                   want_probs=False)
+        torch.cuda.synchronize()
+        got_cut = st[..., 5].cpu().numpy().astype(np.float32)
+        _, ref, _ = oracle.tree_probs(inp, which, want_probs=False)
+        ref_cut = ref[..., 6].astype(np.float32)
+        differs = (got_cut != ref_cut) & rows[None, :]
+        near = (ref[..., 5] < MARGIN) & rows[None, :]
+        assert not (differs & ~near).any(), (
+            f"{int((differs & ~near).sum())} rows cut at another logit although the nucleus boundary is "
+            f"further than 1e-6 from top_p")
+        tally.rows += int(rows.sum()) * B
+        tally.rows_near_boundary += int(near.sum())
+        tally.rows_cut_differs += int(differs.sum())
+        bad_seq |= differs.any(1)
+    tally.sequences_set_aside += int(bad_seq.sum())
+    return bad_seq
 
 
 def compare_decisions(ref, got, parent) -> Tally:
@@ -96,10 +131,21 @@ def run_oracle(batch, algo, want_residual=False):
 
 
 def check_batch(batch, algo, full=True) -> Tally:
-    """Plain call (fast path) and, if ``full``, a call with every optional output, both against the oracle."""
+    """Plain call (fast path) and, if ``full``, a call with every optional output, both against the oracle.
+    With top-k / top-p the rows' cuts are compared first (``settle_cuts``)."""
+    w = batch.workload
+    pre = Tally()
+    if (0 < w.top_k < w.V) or w.top_p < 1.0:
+        bad = settle_cuts(batch, oracle_inputs(batch), pre)
+        if bad.any():
+            batch = batch.select([i for i in range(w.B) if not bad[i]])
+            if batch.workload.B == 0:
+                return pre
     inp, ref = run_oracle(batch, algo, want_residual=full)
     parent = batch.parent.cpu().numpy()
     tally = compare_decisions(ref, gpu_verify(batch, algo), parent)
+    tally.add(pre)
+    tally.sequences += batch.workload.B
     if not full:
         return tally
     got = gpu_verify(batch, algo, residual=True, node_thr=True, features=True, margin=True,

@@ -1,0 +1,38 @@
+"""The five workload configurations at full size, in the launch configuration the benchmark times:
+every sequence of every batch against the CPU oracle -- decisions, tokens, the residual the bonus was
+drawn from, every node's threshold / weight, margins and the selector features.  One tally over all
+configurations bounds the tolerated (near-margin) differences by 1e-4 of all decisions."""
+import pytest
+import torch
+
+from paper_2602_16994_b200.synth import WORKLOADS, make_batch
+from tests.parity import Tally, check_batch
+
+pytestmark = pytest.mark.gpu
+
+TOTAL = Tally()
+CONFIGS = ["cfg1_tiny", "cfg2_llama3_b8", "cfg3_qwen_b32"] + [f"cfg4_gemma_delayed_d{d}" for d in range(5)] + \
+          ["cfg5_serving_b128"]
+
+
+@pytest.mark.parametrize("name", CONFIGS)
+def test_config_full_batch(name):
+    w = WORKLOADS[name]
+    batch = make_batch(w, seed=0, device="cuda")
+    for algo in w.algorithms:
+        t = check_batch(batch, algo, full=True)
+        TOTAL.add(t)
+        print(f"{name} {algo}: {vars(t)}")
+    del batch
+    torch.cuda.empty_cache()
+
+
+def test_tolerated_differences_over_all_configs():
+    """Runs after the configurations above (same module, file order)."""
+    assert TOTAL.decisions > 10000, "the configuration tests did not run before this one"
+    assert TOTAL.near_margin_mismatches < 1e-4 * TOTAL.decisions, vars(TOTAL)
+    # rows the device cut at another logit than the oracle (allowed only where the nucleus boundary is within
+    # 1e-6 of top_p; the sequences that hold one are set aside): fewer than 1e-3 of the rows compared
+    assert TOTAL.rows_cut_differs <= 1e-3 * TOTAL.rows, vars(TOTAL)
+    assert TOTAL.sequences_set_aside <= TOTAL.rows_cut_differs <= TOTAL.rows_near_boundary
+    print(vars(TOTAL))

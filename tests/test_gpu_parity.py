@@ -37,6 +37,12 @@ SHAPES = [
     small("root_only", 3000, "bf16", 1, 0, 0, 3),         # N = 1: just the bonus draw from p
     small("wide", 640, "f32", 16, 0, 1, 3),               # 16 children under one node
     small("cold", 8192, "bf16", 4, 1, 2, 4, sigma=1.2, T=0.3),
+    # near-greedy, nothing truncated, several siblings: target and draft put nearly all their mass on
+    # the same token, so residual masses are tiny differences of probabilities close to 1
+    small("cold_T02", 50000, "bf16", 4, 1, 3, 8, sigma=1.0, T=0.2),
+    small("cold_T015", 50000, "bf16", 4, 1, 3, 8, sigma=0.3, T=0.15),
+    small("cold_T02_f32", 32000, "f32", 6, 0, 2, 6, sigma=0.5, T=0.2),
+    small("cold_T015_v128256", 128256, "bf16", 4, 2, 4, 4, sigma=0.5, T=0.15),
 ]
 
 
@@ -53,24 +59,6 @@ def test_cfg2_full_size(algo):
     batch = make_batch(WORKLOADS["cfg2_llama3_b8"], seed=0, device="cuda")
     t = check_batch(batch, algo, full=True)
     assert t.near_margin_mismatches == 0
-
-
-@pytest.mark.parametrize("algo", ALGOS)
-def test_cfg4_sweep_sampled(algo):
-    """Gemma-sized vocabulary, delayed depth d in {0, 2, 4}: two sampled sequences of the full batch."""
-    for d in (0, 2, 4):
-        w = WORKLOADS[f"cfg4_gemma_delayed_d{d}"]
-        full = make_batch(w, seed=0, device="cuda")
-        got = gpu_verify(full, algo)
-        sub = full.select([3, 11])
-        _, ref = run_oracle(sub, algo)
-        for i, b in enumerate((3, 11)):
-            if got.accepted_node[b].item() != ref.accepted_node[i]:
-                assert min(ref.trace_margins[i], default=1.0) < 1e-6
-            elif got.bonus_token[b].item() != ref.bonus_token[i]:
-                assert ref.bonus_margin[i] < 1e-6
-        del full, sub
-        torch.cuda.empty_cache()
 
 
 @pytest.mark.parametrize("algo", ALGOS)
@@ -263,55 +251,12 @@ TRUNC_SHAPES = [
 ]
 
 
-def _unsure_sequences(inp):
-    """Sequences with a row whose nucleus boundary lies within 1e-6 of top_p (either side may keep or
-    drop the boundary group there)."""
-    _, sp, _ = oracle.tree_probs(inp, 0, want_probs=False)
-    _, sq, _ = oracle.tree_probs(inp, 1, want_probs=False)
-    parent = inp.parent if inp.parent.ndim == 1 else inp.parent[0]
-    internal = np.zeros(parent.shape[0], bool); internal[parent[1:]] = True
-    return (sp[..., 5] < 1e-6).any(1) | (sq[:, internal, 5] < 1e-6).any(1)
-
-
 @pytest.mark.parametrize("algo", ALGOS)
 @pytest.mark.parametrize("w", TRUNC_SHAPES, ids=lambda w: w.name)
 def test_truncated_verification(algo, w):
     batch = make_batch(w, seed=2, device="cuda")
-    inp = oracle_inputs(batch)
-    unsure = _unsure_sequences(inp)
-    assert unsure.mean() < 0.5
-    keep = [i for i in range(w.B) if not unsure[i]]
-    check_batch(batch.select(keep), algo)
-
-
-def test_cfg3_and_cfg5_sampled():
-    """The truncating workloads at full size in the bench's launch configuration; sampled sequences
-    against the oracle (SpecInfer + bonus, cfg5 with the selector features)."""
-    for name, picks in (("cfg3_qwen_b32", [0, 13, 31]), ("cfg5_serving_b128", [5, 77])):
-        w = WORKLOADS[name]
-        full = make_batch(w, seed=0, device="cuda")
-        got = binding.verify_specinfer(full.target_logits, full.draft_logits, full.parent, full.token, full.u_accept,
-                                       full.u_bonus, w.temperature, w.top_k, w.top_p, features=w.features)
-        torch.cuda.synchronize()
-        assert (got.status.cpu().numpy() == 0).all()
-        sub = full.select(picks)
-        inp, ref = run_oracle(sub, "specinfer")
-        unsure = _unsure_sequences(inp)
-        for i, b in enumerate(picks):
-            if unsure[i]:
-                continue
-            if got.accepted_node[b].item() != ref.accepted_node[i]:
-                assert min(ref.trace_margins[i], default=1.0) < 1e-6
-            elif got.bonus_token[b].item() != ref.bonus_token[i]:
-                assert ref.bonus_margin[i] < 1e-6
-            else:
-                np.testing.assert_array_equal(got.out_tokens[b].cpu().numpy(), ref.out_tokens[i])
-        if w.features:
-            _, sp, _ = oracle.tree_probs(inp, 0, want_probs=False)
-            f = got.node_features.cpu().numpy()[picks].astype(np.float64)
-            assert np.abs(f[..., 0] - sp[..., 3]).max() < 1e-4 and np.abs(f[..., 2] - sp[..., 4]).max() < PROB_TOL
-        del full, sub
-        torch.cuda.empty_cache()
+    t = check_batch(batch, algo)
+    assert t.sequences_set_aside == 0, vars(t)
 
 
 def test_traversal_weight_one_with_a_vanishing_residual():
