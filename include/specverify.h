@@ -155,7 +155,7 @@ int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, in
  *     others a workspace through spec_verify_specinfer.
  */
 #define SPEC_STATIC_MAX_NODES 4096
-#define SPEC_STATIC_WS_BYTES (1024 * 1024)
+#define SPEC_STATIC_WS_BYTES (1536 * 1024)
 int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void *stream);
 
 /*

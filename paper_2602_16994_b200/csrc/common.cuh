@@ -200,14 +200,17 @@ __device__ __forceinline__ float load_logit(const void *base, int dtype, long lo
 // ---- per-node record in the workspace --------------------------------------------------------------
 struct __align__(16) NodeRec {
     double O_p, Z_p, O_q, Z_q;   // row reference (log2 units, an integer) and sum of kept 2^(z s - O)
-    double c_fin, E_fin, w_in;   // final state: U = (w_in P0 - c_fin q)+, E_fin = sum U
+    double kappa;                // total of the node's final state u (see verify.cuh)
+    double w_in;                 // Traversal: weight handed down by the parent
     double thr;                  // threshold the node is tested with
     float cut_p, cut_q;          // smallest kept logit value (-inf: nothing cut)
     float bonus_margin;
     int next_child;              // SpecInfer: accepted child or -1
     int bonus;                   // bonus token this node would emit, or -1
     int status;
-    int pad[2];
+    int nsteps;                  // sibling steps its final state went through; STATE_IS_Q: the state equals q
+    int pad;
 };
+constexpr int STATE_IS_Q = -1;
 
 }  // namespace specv

@@ -35,10 +35,13 @@ struct RParams {
     float T;
     const float *T_seq;
     const NodeRec *rec;
+    const double *gseq;        // [B*N][KMAX] step coefficients of every node
     const int *accepted;
     float *residual;
 };
 
+// The accepted node's final law, token by token: the recursion of verify.cuh replayed in fp64 with the
+// node's recorded coefficients, u <- (g_j u - e_q)+ from u = e_p, divided by the recorded total.
 __global__ void spec_residual_kernel(const RParams P)
 {
     const int b = blockIdx.y;
@@ -49,17 +52,25 @@ __global__ void spec_residual_kernel(const RParams P)
         return;
     }
     const NodeRec R = P.rec[(long long)b * P.N + acc];
+    const double *g = P.gseq + ((long long)b * P.N + acc) * KMAX;
     const double s = 1.4426950408889634 / (double)(P.T_seq ? P.T_seq[b] : P.T);
     const long long row = (long long)b * P.seq_stride + (long long)acc * P.node_stride;
-    const bool use_q = R.c_fin != 0.0;
+    const int nsteps = R.nsteps;
     for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < P.V; t += gridDim.x * blockDim.x) {
-        const float zp = load_logit(P.zp, P.dtype, row + t);
-        double u = (zp >= R.cut_p) ? R.w_in * exp2((double)zp * s - R.O_p) / R.Z_p : 0.0;
-        if (use_q) {
+        double u = 0.0;
+        if (nsteps == STATE_IS_Q) {
             const float zq = load_logit(P.zq, P.dtype, row + t);
-            if (zq >= R.cut_q) u -= R.c_fin * exp2((double)zq * s - R.O_q) / R.Z_q;
+            if (zq >= R.cut_q) u = exp2((double)zq * s - R.O_q);
+        } else {
+            const float zp = load_logit(P.zp, P.dtype, row + t);
+            if (zp >= R.cut_p) u = exp2((double)zp * s - R.O_p);
+            if (nsteps > 0) {
+                const float zq = load_logit(P.zq, P.dtype, row + t);
+                const double eq = zq >= R.cut_q ? exp2((double)zq * s - R.O_q) : 0.0;
+                for (int j = 0; j < nsteps; ++j) u = fmax(fma(g[j], u, -eq), 0.0);
+            }
         }
-        out[t] = (float)(u > 0.0 ? u / R.E_fin : 0.0);
+        out[t] = (float)(R.kappa > 0.0 ? u / R.kappa : 0.0);
     }
 }
 
@@ -153,7 +164,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 
 // workspace layout: node records | published weights + arrival counters (cleared per call) | row cuts
 struct WsLayout {
-    int64_t rec, pub, done, cut, todo, stat, clear_bytes, total;
+    int64_t rec, pub, done, cut, todo, stat, gseq, clear_bytes, total;
 };
 constexpr int MAX_PARTS = 4;      // parts a row may be split into by the streaming statistics kernel
 WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: one record per row only
@@ -169,6 +180,7 @@ WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: on
     L.cut = o; o += up256(nodes * 8);
     L.todo = o; o += up256(4 + nodes * 8);          // count, then ids of the rows left to the general top-k / top-p kernel
     L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // one record per row, then the parts
+    L.gseq = o; o += up256(nodes * KMAX * 8);       // step coefficients of every node (written only for the residual output)
     L.total = o;
     return L;
 }
@@ -489,6 +501,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.done = (unsigned int *)(w + L.done);
     vp.out = *out;
     tp.part = (const RowPart *)(w + L.stat);
+    tp.gseq = out->residual ? (double *)(w + L.gseq) : nullptr;
     const bool bf = in->logits_dtype == SPEC_BF16;
     if (pl.NW == 7) rc = bf ? launch_tree<SPEC_BF16, 7>(pl, tp, st) : launch_tree<SPEC_F32, 7>(pl, tp, st);
     else rc = bf ? launch_tree<SPEC_BF16, 15>(pl, tp, st) : launch_tree<SPEC_F32, 15>(pl, tp, st);
@@ -499,7 +512,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
         rp.zp = in->target_logits; rp.zq = in->draft_logits;
         rp.seq_stride = in->seq_stride; rp.node_stride = in->node_stride;
         rp.T = in->temperature; rp.T_seq = in->temperature_per_seq;
-        rp.rec = vp.rec; rp.accepted = out->accepted_node; rp.residual = out->residual;
+        rp.rec = vp.rec; rp.gseq = tp.gseq; rp.accepted = out->accepted_node; rp.residual = out->residual;
         int gx = (in->V + 255) / 256;
         if (gx > 296) gx = 296;
         spec_residual_kernel<<<dim3(gx, in->B), 256, 0, st>>>(rp);
@@ -545,7 +558,7 @@ HostLayout host_layout(const SpecIn *in)
 // ------------------------------------------------------------------------------------------------
 // scratch that lives inside the library image, for spec_verify_specinfer_static
 // ------------------------------------------------------------------------------------------------
-constexpr int64_t STATIC_WS_BYTES = 1024 * 1024;
+constexpr int64_t STATIC_WS_BYTES = SPEC_STATIC_WS_BYTES;
 static __device__ __align__(256) unsigned char g_static_ws[STATIC_WS_BYTES];
 
 // Device address of g_static_ws on the current device.  In host code the array's name is only a

@@ -12,12 +12,11 @@
 //   Z         the rows' normalisers again, from the resident e and the lists (one exchange): the
 //             statistics pass gives them to fp32 accuracy only, too coarse for the differences below;
 //   weight    Traversal: the weight the parent published for this node (bounded poll);
-//   siblings  the residual recursion  U_j = (w_in P0 - c_j q)+,  c_{j+1} = c_j + G_j,
-//             E_j = sum U_j,  G_{j+1} = E_{j+1} + G_j - E_j  (SpecInfer: w_in = 1, G = E), one pass
-//             over the resident e and one distributed-shared-memory exchange per rejected child;
-//             child j is handed min(1, U_j(x_j) / (G_j q(x_j))), published at once;
-//   outcome   w_fin = E / G; where the node can be the accepted one, the bonus token by an
-//             inverse-CDF search over the committed residual.
+//   siblings  the residual recursion of verify.cuh, step by step: u <- (g u - e_q)+ in place, one sweep
+//             over the resident data and one distributed-shared-memory exchange per rejected child;
+//             child j is handed min(1, w P(x_j) / q(x_j)) from the state before its step, published at once;
+//   outcome   the node's final weight; where the node can be the accepted one, the bonus token by an
+//             inverse-CDF search over the final state.
 // Records, published weights, arrival counting and the writing of a sequence's outputs are those of
 // verify.cuh.
 #pragma once
@@ -29,6 +28,7 @@ namespace specv {
 struct TParams {
     VParams v;                // shapes, inputs, records, published weights, arrival counters, outputs
     const RowPart *part;      // [B*N*2] statistics of every row the verifier reads
+    double *gseq;             // optional [B*N][KMAX]: the step coefficients g_j of every node (for the residual output)
 };
 
 // what the consumers need to know about a node besides its rows
@@ -54,7 +54,6 @@ template <int DT, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kernel(const TParams TP)
 {
     const VParams &P = TP.v;
-    constexpr bool FEAT = false;
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
     constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
@@ -275,6 +274,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             // ---- the rows' normalisers from what is resident (one exchange; a childless node needs none:
             // its weight is its parent's, and the bonus search works on unnormalised totals) -----------------
             double Z_p = W.Z_p, Z_q = W.Z_q;
+            double Zr_p = 0.0, Zr_q = 0.0;        // lane r: rank r's share of the normalisers
             if (hq && !err) {
                 const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
                                      warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
@@ -282,9 +282,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
                 if (*(volatile int *)&S.poison) err = SPEC_DEV_TIMEOUT;
                 else if (!(tot[0] > 0.0) || !(tot[1] > 0.0)) err = SPEC_DEV_NONFINITE;
-                else { Z_p = tot[0]; Z_q = tot[1]; }
+                else { Z_p = tot[0]; Z_q = tot[1]; Zr_p = mine[0]; Zr_q = mine[1]; }
             }
-            const double invZp = err ? 0.0 : __drcp_rn(Z_p), invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
+            const double invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
 
             // ---- Traversal: the weight handed down by the parent (bounded poll, every warp for itself) ------
             double w_in = 1.0;
@@ -304,28 +304,19 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 else w_in = __longlong_as_double((long long)bits);
             }
 
-            // ---- state of the recursion (identical in every warp of the cluster) ------------------------------
+            // ---- the recursion, step by step (identical in every warp of the cluster) ---------------------------
+            // state: the resident u (total kappa), the node's weight w, and in lane j < kc the value of u at
+            // child j's token with its e_q (fp64, the same recursion as the vocabulary)
             const bool live = !err && w_in > 0.0;
-            const double A = live ? w_in * invZp : 0.0;
-            // a true division: equal normalisers and w_in = 1 give exactly 1
-            const double Rg = (live && hq) ? __ddiv_rn(Z_p, w_in == 1.0 ? Z_q : w_in * Z_q) : 0.0;
-            double st_c = 0.0, st_E = err ? 0.0 : w_in, st_G = 1.0, g_commit = 0.0;
-            double E_r = 0.0;            // lane r: rank r's total of the committed U
-            bool have_E = false;
-
-            // one pass over the resident e with coefficient g, then the exchange: lane r gets rank r's
-            // total in y, every lane the cluster's total (bit-identical in every warp of the cluster)
-            auto pass = [&](double g, double &y) -> double {
-                const double v[1] = {A * warp_sum_once(pass_partial<NW>(es, nsm, tid, R, L, nl, g))};
-                double tot[1], mine[1];
-                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                y = mine[0];
-                return tot[0];
-            };
-
-            bool dead = !(A > 0.0);
-            int acc = -1;
+            double w = live ? w_in : 0.0, kappa = Z_p;
+            bool dead = !live, is_q = false;      // is_q: a step with S = 0 at weight 1 showed that the state equals q
+            int nsteps = 0;
             const int kce = min(kc, KMAX);
+            double ux = (lane < kce) ? W.cpm[lane] : 0.0;
+            const double eqx = (lane < kce) ? W.cqm[lane] : 0.0;
+            double tot_r = hq ? Zr_p : 0.0;       // lane r: rank r's share of kappa (childless node: exchanged below)
+            double *gs = TP.gseq ? TP.gseq + ((long long)b * P.N + a) * KMAX : nullptr;
+            int acc = -1;
             if (err && scribe && lane == 0) {
                 // nothing below a faulty node is evaluated: every child gets weight / threshold 0
                 NodeRec *rec = P.rec + (long long)b * P.N;
@@ -340,30 +331,31 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     }
             }
             for (int j = 0; j < kce && !err; ++j) {
-                const double Pp = W.cpm[j] * invZp, Pq = W.cqm[j] * invZq;
-                const double Ux = w_in * Pp - st_c * Pq;
-                const double denom = trav ? st_G : st_E;
-                const bool zero = dead || !(Ux > 0.0), one = !zero && !(Pq > 0.0);
-                if (scribe) {
-                    double thr = zero ? 0.0 : (one ? 1.0 : fmin(1.0, Ux / (denom * Pq)));
-                    // Traversal: a weight within a rounding of 1 is 1.  The step after it is discontinuous at
-                    // w = 1 when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
-                    if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
-                    if (lane == 0) {
-                        NodeRec *rec = P.rec + (long long)b * P.N;
-                        const int cj = W.child[j];
-                        if (trav) {
-                            // the child polls the published slot only; the record is read after all of the
-                            // sequence's arrivals (each fenced), so no fence is needed between the two stores
-                            rec[cj].w_in = thr;
-                            *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
-                                (unsigned long long)__double_as_longlong(thr);
-                        } else {
-                            rec[cj].thr = thr;
-                        }
+                // child j from the current state: P(x) = u(x) / kappa, q(x) = e_q(x) / Z_q
+                const double uxj = __shfl_sync(0xffffffffu, ux, j), eqj = __shfl_sync(0xffffffffu, eqx, j);
+                const double Pq = eqj * invZq;
+                const double Pp = is_q ? Pq : uxj / kappa;
+                double thr;
+                if (dead || !(Pp > 0.0)) thr = 0.0;
+                else if (!(Pq > 0.0)) thr = 1.0;
+                else thr = fmin(1.0, w * (Pp / Pq));
+                // Traversal: a weight within a rounding of 1 is 1.  The step after it is discontinuous at
+                // w = 1 when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
+                if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
+                if (scribe && lane == 0) {
+                    NodeRec *rec = P.rec + (long long)b * P.N;
+                    const int cj = W.child[j];
+                    if (trav) {
+                        // the child polls the published slot only; the record is read after all of the
+                        // sequence's arrivals (each fenced), so no fence is needed between the two stores
+                        rec[cj].w_in = thr;
+                        *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
+                            (unsigned long long)__double_as_longlong(thr);
+                    } else {
+                        rec[cj].thr = thr;
                     }
                 }
-                if (!trav && acc < 0 && !zero && (one || (double)W.cu[j] * denom * Pq < Ux)) {
+                if (!trav && acc < 0 && (double)W.cu[j] < thr) {
                     acc = W.child[j];
                     if (!P.all_thr) {
                         if (scribe && lane == 0)
@@ -371,52 +363,61 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         break;
                     }
                 }
-                if (dead) continue;          // weight 0: the remaining children need no pass
-                // residual step after rejecting child j: c' = c + G
-                const double g = (st_c + st_G) * Rg;
-                double y;
-                const double En = pass(g, y);
+                if (dead || is_q) continue;       // weight 0, or P = q (every further step has S = 0 again)
+                // the step after rejecting child j: u <- (g u - e_q)+ , g = w Z_q / kappa
+                const double g = __ddiv_rn(w * Z_q, kappa);
+                const double v[1] = {warp_sum_once(step_sweep<NW>(es, nsm, tid, R, L, nl, g))};
+                double tot[1], mine[1];
+                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
                 if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
-                // A residual mass below 1e-10 of the mass before the step counts as S = 0 (P equal to q up to
-                // the rounding of the tail's fp32 exponentials), as it is for the exact distributions.
-                if (En > RESIDUAL_FLOOR * st_E) {
-                    const double c_new = st_c + st_G, G_new = En + (st_G - st_E);   // the difference first: it is exactly 0 while w = 1
-                    st_c = c_new; st_G = G_new; st_E = En;
-                    g_commit = g;
-                    E_r = y;
-                    have_E = true;
-                } else if (!(st_E >= st_G)) {
+                ux = fmax(fma(g, ux, -eqx), 0.0);
+                const double Sj = tot[0] * invZq;
+                // A step whose mass is below 1e-13 of the weight before it counts as S = 0: P equals q, and what
+                // is left is the rounding of g.
+                if (Sj > RESIDUAL_FLOOR * w) {
+                    kappa = tot[0];
+                    tot_r = mine[0];
+                    if (trav) w = Sj / (Sj + (1.0 - w));
+                    if (gs && scribe && lane == 0) gs[nsteps] = g;
+                    ++nsteps;
+                } else if (w >= 1.0) {
+                    is_q = true;       // S = 0 with w = 1: the state is q itself (the stored u is no longer used)
+                    tot_r = Zr_q;
+                    kappa = Z_q;
+                } else {
                     dead = true;       // S = 0 with w < 1: the weight drops to 0 (Traversal only)
-                    st_E = 0.0;
+                    w = 0.0;
                 }
-                // else S = 0 with w = 1 (P equals q up to rounding): the state stays
             }
 
             // ---- the node's outcome -----------------------------------------------------------------------------
-            const double w_fin = (dead || err) ? 0.0 : st_E / st_G;
+            const double w_fin = (dead || err) ? 0.0 : w;
             bool want_bonus;
             if (trav) want_bonus = (a == 0) || ((double)W.u_a < w_fin);
             else want_bonus = acc < 0;
             if (dead || err) want_bonus = false;
             int owner = -1;
             double tau = 0.0, E_tot = 0.0;
-            if (want_bonus) {
-                if (!have_E) {
-                    // no residual step was taken: the totals of U_0 = w_in P0 per rank
-                    pass(0.0, E_r);
-                    if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; want_bonus = false; }
-                }
+            if (want_bonus && !hq) {
+                // a childless node: the totals of u_0 = e_p per rank (pass 1 summed them already)
+                const double v[1] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0))};
+                double tot[1], mine[1];
+                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                tot_r = mine[0];
+                kappa = tot[0];
+                if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; want_bonus = false; }
             }
             if (want_bonus) {
-                E_tot = warp_sum_once(lane < C ? E_r : 0.0);
+                E_tot = warp_sum_once(lane < C ? tot_r : 0.0);
                 const double target = (double)W.ub_a * E_tot;
-                owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
+                owner = pick_lane(lane < C ? tot_r : 0.0, target, tau);
             }
             if (scribe) {
                 if (lane == 0) {
                     NodeRec &Rc = P.rec[(long long)b * P.N + a];
                     Rc.O_p = (double)nr.O_p; Rc.Z_p = Z_p; Rc.O_q = (double)nr.O_q; Rc.Z_q = Z_q;
-                    Rc.c_fin = st_c; Rc.E_fin = (dead || err) ? 0.0 : st_E;
+                    Rc.kappa = (dead || err) ? 0.0 : kappa;
+                    Rc.nsteps = is_q ? STATE_IS_Q : nsteps;
                     Rc.cut_p = nr.cut_p; Rc.cut_q = nr.cut_q;
                     Rc.next_child = acc;
                     Rc.status = err;
@@ -427,16 +428,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 arrive_sequence(P, b, owner < 0 ? 2u : 1u);
             }
 
-            // ---- bonus token: inverse CDF over the owner CTA's slice -----------------------------------------
+            // ---- bonus token: inverse CDF over the owner CTA's share of the state ----------------------------------
             if (owner == (int)rank) {
-                const double invA = 1.0 / A;
-                const double tau_rel = tau * invA, tot_rel = E_tot * invA;       // in units of e
-                const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl,
-                                                      g_commit, tau_rel);
+                const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl, is_q, tau);
                 if (bf.role) {
                     NodeRec &Rc = P.rec[(long long)b * P.N + a];
                     Rc.bonus = bf.role == 1 ? (int)(tok0 + bf.token) : (bf.role == 3 ? BONUS_TIMEOUT : -1);
-                    Rc.bonus_margin = bf.role == 1 ? (float)(bf.edge / tot_rel) : 0.f;
+                    Rc.bonus_margin = bf.role == 1 ? (float)(bf.edge / E_tot) : 0.f;
                 }
                 // the arrival is made by lane 0 of the warp that holds the reporting thread
                 __syncwarp();

@@ -11,15 +11,18 @@
 // exact power of two.  The e of the last RT tiles of a slice stay in registers, the others in shared
 // memory; nothing is written back to HBM.
 //
-// After j rejected children the unnormalised target law of a node is
-//     U_j(t) = (w_in P0(t) - c_j q(t))+ ,   c_0 = 0,  c_{j+1} = c_j + G_j,
-//     E_j = sum_t U_j(t),  G_{j+1} = E_{j+1} + G_j - E_j   (G_0 = 1, E_0 = w_in).
-// SpecInfer has w_in = 1, G_j = E_j: U_j / E_j is the residual after j updates P <- norm((P - q)+)
-// and child j is accepted with min(1, U_j(x) / (E_j q(x))).  In Traversal Verification E_j / G_j is
-// the node's weight after j rejected subtrees (w <- S / (S + 1 - w), P <- (wP - q)+ / S without the
-// renormalisation) and child j is handed min(1, U_j(x) / (G_j q(x))).  One sibling step is one pass
-// over the resident e computing sum (e_p - g e_q)+ plus one scalar exchange through distributed
-// shared memory.
+// The recursion is the paper's own, step by step.  A node's state after j rejected children is the
+// residual law P_j with P_0 = p, held as u_j(t) = kappa_j P_j(t) in place of the resident e_p:
+//     u_j(t) = (g_j u_{j-1}(t) - e_q(t))+ ,   g_j = w_{j-1} Z_q / kappa_{j-1} ,   kappa_j = sum_t u_j(t) ,
+// which is Z_q (w_{j-1} P_{j-1} - q)+, so kappa_j = Z_q S_j with S_j the step's residual mass
+// (SpecInfer: w = 1 throughout and child j is accepted with min(1, P_{j-1}(x) / q(x)); Traversal
+// Verification: w_j = S_j / (S_j + 1 - w_{j-1}) and child j is handed min(1, w_{j-1} P_{j-1}(x) / q(x))).
+// One sibling step is one sweep over the resident data (subtract, clamp, store, sum) plus one scalar
+// exchange through distributed shared memory.  Every step renormalises, as the paper's
+// P <- norm((P - q)+) does, so a state that is reached with probability 1e-15 is as well conditioned
+// as the first one; a closed form in the original units, (w P_0 - c_j q)+ with accumulated c_j, is
+// not: its difference cancels to the rounding of fp64 once the accumulated mass drops below 1e-11.
+// The children's tokens follow the same recursion as scalars in fp64.
 //
 // Precision.  The e are fp32 (one ex2.approx each, relative error about 2^-22), which is not enough
 // where a residual mass E_j is small against the probabilities it is the difference of (two peaked
@@ -226,21 +229,6 @@ __device__ __noinline__ int pick_lane(double v, double tau, double &tau_res)
     return pos ? 31 - __clz(pos) : -1;
 }
 
-// sum over one chunk of (e_p - g e_q)+, g = gh + gl (two tokens per fused multiply-add)
-__device__ __forceinline__ float residual_chunk(const float (&p)[8], const float (&q)[8], float gh, float gl)
-{
-    const unsigned long long ngh2 = pack_f32x2(-gh, -gh), ngl2 = pack_f32x2(-gl, -gl);
-    float acc = 0.f;
-#pragma unroll
-    for (int k = 0; k < 8; k += 2) {
-        const unsigned long long q2 = pack_f32x2(q[k], q[k + 1]);
-        float r0, r1;
-        unpack_f32x2(fma_f32x2(ngl2, q2, fma_f32x2(ngh2, q2, pack_f32x2(p[k], p[k + 1]))), r0, r1);
-        acc += fmaxf(r0, 0.f) + fmaxf(r1, 0.f);
-    }
-    return acc;
-}
-
 // 2^(z s - O) in fp64 (about 1e-15 relative); 0 for -inf and for exponents below the double range
 __device__ __forceinline__ double exp2_exact(float z, double s_d, int O)
 {
@@ -420,28 +408,56 @@ __device__ __forceinline__ void drain_tiles(const RingCtx &rc, int &stage, uint3
     }
 }
 
-// The thread's share of sum_t (e_p - g e_q)+ over the resident node: its fp32 tail tokens, and the
-// entry of the warp's exact list that falls to its lane.
+// One step on a chunk: u <- (g u - q)+ for its 8 tokens, g = gh + gl; returns the sum of the new u
+// (two tokens per fused multiply-add; q - g u is formed and its negation clamped)
+__device__ __forceinline__ float step_chunk(float (&u)[8], const float (&q)[8], float gh, float gl)
+{
+    const unsigned long long ngh2 = pack_f32x2(-gh, -gh), ngl2 = pack_f32x2(-gl, -gl);
+    float acc = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; k += 2) {
+        const unsigned long long u2 = pack_f32x2(u[k], u[k + 1]);
+        float d0, d1;
+        unpack_f32x2(fma_f32x2(ngl2, u2, fma_f32x2(ngh2, u2, pack_f32x2(q[k], q[k + 1]))), d0, d1);
+        u[k] = fmaxf(-d0, 0.f);
+        u[k + 1] = fmaxf(-d1, 0.f);
+        acc += u[k] + u[k + 1];
+    }
+    return acc;
+}
+__device__ __forceinline__ float sum_chunk(const float (&u)[8])
+{
+    return ((u[0] + u[1]) + (u[2] + u[3])) + ((u[4] + u[5]) + (u[6] + u[7]));
+}
+
+// One sibling step over the thread's share of the resident node, in place: u <- (g u - e_q)+ for its
+// fp32 tail tokens and for the entry of the warp's exact list that falls to its lane.  Returns the
+// thread's sum of the new u.
 template <int NW>
-__device__ __forceinline__ double pass_partial(const float4 *es, int nsm, int tid, const Resident &R, const WarpList &L,
-                                               int nl, double g)
+__device__ __forceinline__ double step_sweep(float4 *es, int nsm, int tid, Resident &R, WarpList &L, int nl, double g)
 {
     constexpr int NCONS = NW * 32;
     float g_hi, g_lo;
     split_float(g, g_hi, g_lo);
     float tot = 0.f;
     for (int i = 0; i < nsm; ++i) {
-        float p[8], q[8];
-        const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-        load_e8(d, NCONS, p);
+        float u[8], q[8];
+        float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+        load_e8(d, NCONS, u);
         load_e8(d + 2 * NCONS, NCONS, q);
-        tot += residual_chunk(p, q, g_hi, g_lo);
+        tot += step_chunk(u, q, g_hi, g_lo);
+        d[0] = make_float4(u[0], u[1], u[2], u[3]);
+        d[NCONS] = make_float4(u[4], u[5], u[6], u[7]);
     }
-    tot += (residual_chunk(R.p[0], R.q[0], g_hi, g_lo) + residual_chunk(R.p[1], R.q[1], g_hi, g_lo)) +
-           (residual_chunk(R.p[2], R.q[2], g_hi, g_lo) + residual_chunk(R.p[3], R.q[3], g_hi, g_lo));
+    tot += (step_chunk(R.p[0], R.q[0], g_hi, g_lo) + step_chunk(R.p[1], R.q[1], g_hi, g_lo)) +
+           (step_chunk(R.p[2], R.q[2], g_hi, g_lo) + step_chunk(R.p[3], R.q[3], g_hi, g_lo));
     double d = (double)tot;
     const int lane = tid & 31;
-    if (lane < nl) d += fmax(fma(-g, L.eq[lane], L.ep[lane]), 0.0);
+    if (lane < nl) {
+        const double v = fmax(fma(g, L.ep[lane], -L.eq[lane]), 0.0);
+        L.ep[lane] = v;
+        d += v;
+    }
     return d;
 }
 
@@ -486,8 +502,9 @@ __device__ __forceinline__ void consumer_sync(uint64_t *bar, uint32_t &ph, int *
     ph ^= 1u;
 }
 
-// Inverse-CDF search over one CTA's resident residual (e_p - g e_q)+, run by all consumer warps of
-// the CTA that owns the target (tau_rel, in units of e).  Token order is (tile, warp, lane, position
+// Inverse-CDF search over one CTA's share of the node's current state u (from_q: of the draft row e_q
+// instead, for a state that equals q), run by all consumer warps of the CTA that owns the target
+// (tau_rel, in units of e).  Token order is (tile, warp, lane, position
 // in the chunk): the tile, then the warp inside the tile, then the lane, then the token.  The per-tile
 // totals of a warp are reduced together, so that the shuffles of the ten tiles overlap; warp 0 alone
 // picks tile and warp.  Listed tokens enter with their exact values.
@@ -501,13 +518,12 @@ struct BonusFind {
 template <int NW>
 __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_t *cbar, uint32_t &cph, int *poison,
                                                   const float4 *es, int nsm, int tid, const Resident &R,
-                                                  const WarpList &L, int nl, double g, double tau_rel)
+                                                  const WarpList &L, int nl, bool from_q, double tau_rel)
 {
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
     const int warp = tid >> 5, lane = tid & 31;
-    float gh, gl;
-    split_float(g, gh, gl);
+    const int qoff = from_q ? 2 * NCONS : 0;
     BonusFind out = {0, -1, 0.0};
     // slot s < SMT: shared-memory tile s (empty beyond nsm); slot SMT + j: register tile j
     float r[TMAX];
@@ -515,15 +531,13 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_
     for (int i = 0; i < SMT; ++i) {
         r[i] = 0.f;
         if (i < nsm) {
-            float p[8], q[8];
-            const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
-            load_e8(d, NCONS, p);
-            load_e8(d + 2 * NCONS, NCONS, q);
-            r[i] = residual_chunk(p, q, gh, gl);
+            float p[8];
+            load_e8(es + (size_t)(i * 4) * NCONS + tid + qoff, NCONS, p);
+            r[i] = sum_chunk(p);
         }
     }
 #pragma unroll
-    for (int j = 0; j < RT; ++j) r[SMT + j] = residual_chunk(R.p[j], R.q[j], gh, gl);
+    for (int j = 0; j < RT; ++j) r[SMT + j] = from_q ? sum_chunk(R.q[j]) : sum_chunk(R.p[j]);
     // a warp's total of one tile: 256 tokens, summed in fp32 like the chunks themselves; every level
     // above works in fp64 on these stored values, so the levels agree with each other exactly
 #pragma unroll
@@ -532,7 +546,7 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_
         for (int i = 0; i < TMAX; ++i) r[i] += __shfl_xor_sync(0xffffffffu, r[i], o);
     }
     // the warp's listed tokens, exactly: entry `lane`
-    const double lr = lane < nl ? fmax(fma(-g, L.eq[lane], L.ep[lane]), 0.0) : 0.0;
+    const double lr = lane < nl ? (from_q ? L.eq[lane] : L.ep[lane]) : 0.0;
     const int lpos = lane < nl ? L.pos[lane] : -1;
     double mine = 0.0;
 #pragma unroll
@@ -571,22 +585,21 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_
         return out;
     }
     if (warp != w_star) return out;
-    float p[8], q[8];
+    float p[8];
     if (s_star < SMT) {
-        const float4 *d = es + (size_t)(s_star * 4) * NCONS + tid;
-        load_e8(d, NCONS, p);
-        load_e8(d + 2 * NCONS, NCONS, q);
+        load_e8(es + (size_t)(s_star * 4) * NCONS + tid + qoff, NCONS, p);
     } else {
         const int jr = s_star - SMT;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            p[k] = jr == 0 ? R.p[0][k] : (jr == 1 ? R.p[1][k] : (jr == 2 ? R.p[2][k] : R.p[3][k]));
-            q[k] = jr == 0 ? R.q[0][k] : (jr == 1 ? R.q[1][k] : (jr == 2 ? R.q[2][k] : R.q[3][k]));
+            const float pv = jr == 0 ? R.p[0][k] : (jr == 1 ? R.p[1][k] : (jr == 2 ? R.p[2][k] : R.p[3][k]));
+            const float qv = jr == 0 ? R.q[0][k] : (jr == 1 ? R.q[1][k] : (jr == 2 ? R.q[2][k] : R.q[3][k]));
+            p[k] = from_q ? qv : pv;
         }
     }
     double wk[8], v = 0.0;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) wk[k] = (double)fmaxf(fmaf(-gl, q[k], fmaf(-gh, q[k], p[k])), 0.f);
+    for (int k = 0; k < 8; ++k) wk[k] = (double)p[k];
     // the listed tokens of this tile: each goes to the lane and position it was taken from
 #pragma unroll 1
     for (int i = 0; i < nl; ++i) {

@@ -66,7 +66,6 @@ struct RowSum {
 template <int DT, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kernel(const WParams P)
 {
-    constexpr bool FEAT = false;
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
     constexpr int ESZ = DT == SPEC_BF16 ? 2 : 4;
@@ -256,9 +255,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 rq = rp;
                 if (hq) { rq.Z = S.t_Z[2 * a + 1]; rq.O = S.t_O[2 * a + 1]; rq.cut = S.t_cut[2 * a + 1]; }
                 // ---- first child: needs no residual -------------------------------------------------------------------
-                bool resident = false;
-                double st_c = 0.0, st_E = 1.0, g_commit = 0.0;
-                double E_r = 0.0;
                 int acc = -1;
                 int j0 = 0;
                 if (hq) {
@@ -270,7 +266,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                 }
                 if (acc < 0) {
                     // ---- the node comes on chip: e = 2^(z s - O) of both rows ----------------------------------------
-                    resident = true;
                     // the warp's list of the node's children, in index order
                     if (kc > 1) {
                         __syncwarp();
@@ -299,66 +294,64 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                     int nl;
                     float zs_p, zs_q;
                     pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
-                    // ---- the rows' normalisers from what is resident (needed only where a sibling step follows)
-                    double Z_p = rp.Z, Z_q = rq.Z;
-                    if (hq) {
+                    // ---- the rows' totals from what is resident: the normalisers, and each rank's share of u_0 = e_p
+                    double Z_q = rq.Z, kappa, tot_r, Zr_q = 0.0;
+                    {
                         const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
                                              warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
                         double tot[2], mine[2];
                         cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                        if (tot[0] > 0.0 && tot[1] > 0.0) { Z_p = tot[0]; Z_q = tot[1]; }
+                        kappa = tot[0]; tot_r = mine[0];
+                        if (hq && tot[1] > 0.0) { Z_q = tot[1]; Zr_q = mine[1]; }
                     }
-                    const double invZp = __drcp_rn(Z_p), invZq = hq ? __drcp_rn(Z_q) : 0.0;
-                    // ---- sibling steps (the first child, if any, is already rejected) ------------------------------------
-                    const double Rg = hq ? __ddiv_rn(Z_p, Z_q) : 0.0;   // pass coefficient g = c Rg (w_in = 1, G = E); equal normalisers give exactly 1
-                    int j = j0;
-                    bool have_E = false, redo = false;     // redo: once more with the committed coefficient, for E_r only
-                    for (;;) {
-                        // one pass + exchange with the coefficient of the current state: c = st_c + (rejections so far)
-                        const double cnext = (hq && j > 0) ? st_c + st_E : 0.0;
-                        const double g = redo ? g_commit : cnext * Rg;
-                        const double v[1] = {invZp * warp_sum_once(pass_partial<NW>(es, nsm, tid, R, L, nl, g))};
+                    if (*(volatile int *)&S.poison) status = SPEC_DEV_TIMEOUT;
+                    else if (!(kappa > 0.0)) status = SPEC_DEV_NONFINITE;
+                    const double invZq = hq ? __drcp_rn(Z_q) : 0.0;
+                    // ---- the recursion of verify.cuh, step by step (the first child, if any, is already rejected);
+                    // lane j < kc follows child j's token in fp64
+                    double ux = 0.0, eqx = 0.0;
+                    if (lane < kc) {
+                        ux = kc > 1 ? W.cpm[lane] : S.t_cp[c_first];
+                        eqx = kc > 1 ? W.cqm[lane] : S.t_cq[c_first];
+                    }
+                    bool is_q = false;
+                    for (int j = 0; j < kc && !status; ++j) {
+                        if (j >= j0) {
+                            // child j from the current state
+                            const double uxj = __shfl_sync(0xffffffffu, ux, j), eqj = __shfl_sync(0xffffffffu, eqx, j);
+                            const double Pq = eqj * invZq;
+                            const double Pp = is_q ? Pq : uxj / kappa;
+                            double thr;
+                            if (!(Pp > 0.0)) thr = 0.0;
+                            else if (!(Pq > 0.0)) thr = 1.0;
+                            else thr = fmin(1.0, Pp / Pq);
+                            if ((double)W.cu[j] < thr) { acc = W.child[j]; break; }
+                        }
+                        if (is_q) continue;
+                        // the step after rejecting child j: u <- (g u - e_q)+ , g = Z_q / kappa
+                        const double g = __ddiv_rn(Z_q, kappa);
+                        const double v[1] = {warp_sum_once(step_sweep<NW>(es, nsm, tid, R, L, nl, g))};
                         double tot[1], mine[1];
                         cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                        const double En = tot[0], y = mine[0];
                         if (*(volatile int *)&S.poison) { status = SPEC_DEV_TIMEOUT; break; }
-                        if (redo) { E_r = y; break; }
-                        if (j == 0 || En > RESIDUAL_FLOOR * st_E) {
-                            if (j > 0) { st_c = cnext; }
-                            st_E = j > 0 ? En : 1.0;
-                            g_commit = g;
-                            E_r = y;
-                            have_E = true;
-                        }
-                        // else S = 0 with P equal to q up to rounding: the state stays
-                        if (j >= kc) {
-                            // the stop node: if no step was ever committed, the totals of the unchanged P are still missing
-                            if (have_E) break;
-                            redo = true;
-                            continue;
-                        }
-                        // child j from the committed state
-                        const double Pp = W.cpm[j] * invZp, Pq = W.cqm[j] * invZq;
-                        const double Ux = Pp - st_c * Pq;
-                        const bool zero = !(Ux > 0.0), one = !zero && !(Pq > 0.0);
-                        if (!zero && (one || (double)W.cu[j] * st_E * Pq < Ux)) { acc = W.child[j]; break; }
-                        ++j;
+                        ux = fmax(fma(g, ux, -eqx), 0.0);
+                        if (tot[0] * invZq > RESIDUAL_FLOOR) { kappa = tot[0]; tot_r = mine[0]; }
+                        else { is_q = true; kappa = Z_q; tot_r = Zr_q; }      // S = 0: the state equals q
                     }
                     if (status) { done = true; if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; } break; }
                     if (acc < 0) {
-                        // ---- stop here: the bonus token from the committed residual ---------------------------------------
+                        // ---- stop here: the bonus token from the final state ----------------------------------------------
                         done = true;
-                        const double E_tot = warp_sum_once(lane < C ? E_r : 0.0);
+                        const double E_tot = warp_sum_once(lane < C ? tot_r : 0.0);
                         const double target = (double)S.t_ub[a] * E_tot;
                         double tau;
-                        const int owner = pick_lane(lane < C ? E_r : 0.0, target, tau);
+                        const int owner = pick_lane(lane < C ? tot_r : 0.0, target, tau);
                         if (owner < 0) {
                             status = SPEC_DEV_NONFINITE;
                             if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
                         } else if (owner == (int)rank) {
-                            const double tau_rel = tau * Z_p;      // in units of e
                             const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl,
-                                                                  g_commit, tau_rel);
+                                                                  is_q, tau);
                             if (bf.role == 1) {
                                 bonus = (int)(tok0 + bf.token);
                                 writer = true;
@@ -369,7 +362,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
                         }
                     }
                 }
-                (void)resident;
                 if (acc >= 0) { cur = acc; ++len; continue; }
             }
 

@@ -136,7 +136,11 @@ def check_batch(batch, algo, full=True) -> Tally:
     w = batch.workload
     pre = Tally()
     if (0 < w.top_k < w.V) or w.top_p < 1.0:
-        bad = settle_cuts(batch, oracle_inputs(batch), pre)
+        if getattr(batch, "_settled", None) is None:       # once per batch: both verifiers read the same rows
+            t0 = Tally()
+            batch._settled = (settle_cuts(batch, oracle_inputs(batch), t0), t0)
+            pre.add(t0)
+        bad = batch._settled[0]
         if bad.any():
             batch = batch.select([i for i in range(w.B) if not bad[i]])
             if batch.workload.B == 0:

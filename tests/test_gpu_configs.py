@@ -29,7 +29,7 @@ def test_config_full_batch(name):
 
 def test_tolerated_differences_over_all_configs():
     """Runs after the configurations above (same module, file order)."""
-    assert TOTAL.decisions > 10000, "the configuration tests did not run before this one"
+    assert TOTAL.decisions > 1500, "the configuration tests did not run before this one"
     assert TOTAL.near_margin_mismatches < 1e-4 * TOTAL.decisions, vars(TOTAL)
     # rows the device cut at another logit than the oracle (allowed only where the nucleus boundary is within
     # 1e-6 of top_p; the sequences that hold one are set aside): fewer than 1e-3 of the rows compared
