@@ -14,15 +14,15 @@ from dataclasses import dataclass, field
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "spec_oracle.c")
+_SRCS = [os.path.join(_HERE, "spec_oracle.c"), os.path.join(_HERE, "otlp_oracle.c")]
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP over sequences) if the library is missing or stale."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in _SRCS):
         subprocess.check_call(
-            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-o", _LIB, _SRC, "-lm"])
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-o", _LIB] + _SRCS + ["-lm"])
     return _LIB
 
 
@@ -72,6 +72,26 @@ def lib():
         _lib.oracle_sample_bonus.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                              C.c_void_p, C.c_void_p]
         _lib.oracle_max_threads.restype = C.c_int32
+        _lib.oracle_spectr_rho.restype = C.c_double
+        _lib.oracle_spectr_rho.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
+        _lib.oracle_verify_otlp.restype = C.c_int32
+        _lib.oracle_verify_otlp.argtypes = [C.POINTER(_In), C.c_int32] + [C.c_void_p] * 7
+        _lib.oracle_acceptance.restype = C.c_int32
+        _lib.oracle_acceptance.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        _lib.oracle_divergences.restype = C.c_int32
+        _lib.oracle_divergences.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        _lib.oracle_branching.restype = C.c_int32
+        _lib.oracle_branching.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32,
+                                          C.c_void_p]
+        _lib.oracle_block_efficiency.restype = C.c_int32
+        _lib.oracle_block_efficiency.argtypes = [C.POINTER(_In), C.c_int32] + [C.c_void_p] * 4
+        _lib.oracle_node_analysis.restype = C.c_int32
+        _lib.oracle_node_analysis.argtypes = [C.POINTER(_In)] + [C.c_void_p] * 3
+        _lib.oracle_latency_model.restype = C.c_int32
+        _lib.oracle_latency_model.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                              C.c_void_p]
+        _lib.oracle_tps_estimate.restype = C.c_double
+        _lib.oracle_tps_estimate.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
     return _lib
 
 
@@ -239,3 +259,110 @@ def sample_bonus(weights, u):
     if rc:
         raise ValueError(f"oracle_sample_bonus failed with {rc}")
     return tok, mg
+
+
+# ---------------------------------------------------------------------------------------------
+# the other OTLP solvers and the offline analysis (otlp_oracle.c)
+# ---------------------------------------------------------------------------------------------
+SOLVERS = {"nss": 0, "naive": 1, "spectr": 2, "specinfer": 3, "specinfer_uniform": 4}
+
+
+def spectr_rho(p, q, k: int) -> float:
+    p = np.ascontiguousarray(p, np.float64); q = np.ascontiguousarray(q, np.float64)
+    return float(lib().oracle_spectr_rho(_ptr(p), _ptr(q), p.size, int(k)))
+
+
+@dataclass
+class OtlpResult:
+    accepted_node: np.ndarray
+    accept_len: np.ndarray
+    out_tokens: np.ndarray
+    bonus_token: np.ndarray
+    bonus_margin: np.ndarray    # CDF margin of the last residual draw (0: the last token was an accepted child)
+    min_margin: np.ndarray      # smallest |u - threshold| over the acceptance tests made (1: none)
+    status: np.ndarray
+
+
+def verify_otlp(inp: TreeInputs, solver: str) -> OtlpResult:
+    """Top-down verification with NSS / Naive / SpecTr (Algorithms 1-3)."""
+    B, N, _ = inp.shape
+    st = inp.as_struct()
+    acc = np.empty(B, np.int32); alen = np.empty(B, np.int32); toks = np.empty((B, N), np.int32)
+    bonus = np.empty(B, np.int32); bm = np.zeros(B, np.float64); mm = np.ones(B, np.float64)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_verify_otlp(C.byref(st), SOLVERS[solver], _ptr(acc), _ptr(alen), _ptr(toks), _ptr(bonus),
+                                  _ptr(bm), _ptr(mm), _ptr(status))
+    if rc:
+        raise ValueError(f"oracle_verify_otlp failed with {rc}")
+    return OtlpResult(acc, alen, toks, bonus, bm, mm, status)
+
+
+def acceptance(p, q, k: int):
+    """Acceptance rates (Algorithms 6-9): [NSS, Naive, SpecTr, SpecInfer]."""
+    p = np.ascontiguousarray(p, np.float64); q = np.ascontiguousarray(q, np.float64)
+    out = np.empty(4, np.float64)
+    rc = lib().oracle_acceptance(_ptr(p), _ptr(q), p.size, int(k), _ptr(out))
+    if rc:
+        raise ValueError(f"oracle_acceptance failed with {rc}")
+    return out
+
+
+def divergences(p, q):
+    """[L1, KL(p||q), KL(q||p)] in nats."""
+    p = np.ascontiguousarray(p, np.float64); q = np.ascontiguousarray(q, np.float64)
+    out = np.empty(3, np.float64)
+    rc = lib().oracle_divergences(_ptr(p), _ptr(q), p.size, _ptr(out))
+    if rc:
+        raise ValueError(f"oracle_divergences failed with {rc}")
+    return out
+
+
+def branching(solver: str, p, q, xs):
+    """Branching probabilities B(f, xs, xs[i]) (Algorithms 11-14) for every child position."""
+    p = np.ascontiguousarray(p, np.float64); q = np.ascontiguousarray(q, np.float64)
+    x = np.ascontiguousarray(xs, np.int32)
+    out = np.zeros(x.size, np.float64)
+    rc = lib().oracle_branching(SOLVERS[solver], _ptr(p), _ptr(q), p.size, _ptr(x), x.size, _ptr(out))
+    if rc:
+        raise ValueError(f"oracle_branching failed with {rc}")
+    return out
+
+
+def block_efficiency(inp: TreeInputs, solver: str):
+    """(E[tau+1 | tree] float64[B], node_reach [B,N], node_branch [B,N], status) -- equation (3)'s inner sum."""
+    B, N, _ = inp.shape
+    st = inp.as_struct()
+    be = np.zeros(B, np.float64); reach = np.zeros((B, N), np.float64); br = np.zeros((B, N), np.float64)
+    status = np.zeros(B, np.int32)
+    rc = lib().oracle_block_efficiency(C.byref(st), SOLVERS[solver], _ptr(be), _ptr(reach), _ptr(br), _ptr(status))
+    if rc:
+        raise ValueError(f"oracle_block_efficiency failed with {rc}")
+    return be, reach, br, status
+
+
+def node_analysis(inp: TreeInputs):
+    """(acceptance float64[B,N,4], divergences float64[B,N,3], status): NaN at childless nodes."""
+    B, N, _ = inp.shape
+    st = inp.as_struct()
+    acc = np.zeros((B, N, 4), np.float64); dv = np.zeros((B, N, 3), np.float64); status = np.zeros(B, np.int32)
+    rc = lib().oracle_node_analysis(C.byref(st), _ptr(acc), _ptr(dv), _ptr(status))
+    if rc:
+        raise ValueError(f"oracle_node_analysis failed with {rc}")
+    return acc, dv, status
+
+
+def latency_model(t_q, t_p, ctx: int, actions):
+    """Equation (8): forward-pass time of every action (K, L1, L2) at context length ctx."""
+    t_q = np.ascontiguousarray(t_q, np.float64); t_p = np.ascontiguousarray(t_p, np.float64)
+    a = np.ascontiguousarray(actions, np.int32).reshape(-1, 3)
+    out = np.zeros(a.shape[0], np.float64)
+    rc = lib().oracle_latency_model(_ptr(t_q), _ptr(t_p), t_q.size, int(ctx), _ptr(a), a.shape[0], _ptr(out))
+    if rc:
+        raise ValueError(f"oracle_latency_model failed with {rc}")
+    return out
+
+
+def tps_estimate(pi, E, T_hat) -> float:
+    pi = np.ascontiguousarray(pi, np.float64); E = np.ascontiguousarray(E, np.float64)
+    T_hat = np.ascontiguousarray(T_hat, np.float64)
+    return float(lib().oracle_tps_estimate(_ptr(pi), _ptr(E), _ptr(T_hat), pi.size))

@@ -251,13 +251,19 @@ struct NodeRows {
     float thrA_p, thrA_q;     // e above this: always listed (2^-DOM_A of the row's mass)
     float thrB_p, thrB_q;     // e above this: listed while the list has room (2^-DOM_B)
 };
-// Z: the row's normaliser from the statistics pass (fp32 exponentials: good enough for a threshold)
+// Z: the row's normaliser from the statistics pass (fp32 exponentials: good enough for a threshold).
+// The largest e of a row lies in (1/2, 1], so Z > LIST_FLAT_Z means that no token holds more than
+// 1/LIST_FLAT_Z of the row's mass: on such a flat row the second tier would fill with arbitrary tokens
+// at once and buy nothing (small residual masses need two peaked laws), so it is left out.
+constexpr double LIST_FLAT_Z = 16.0;
 __device__ __forceinline__ void set_list_thresholds(NodeRows &nr, double Z_p, double Z_q)
 {
-    nr.thrA_p = (float)(Z_p * (1.0 / (double)(1ull << DOM_A)));
-    nr.thrB_p = (float)(Z_p * (1.0 / (double)(1ull << DOM_B)));
-    nr.thrA_q = nr.hq ? (float)(Z_q * (1.0 / (double)(1ull << DOM_A))) : CUDART_INF_F;
-    nr.thrB_q = nr.hq ? (float)(Z_q * (1.0 / (double)(1ull << DOM_B))) : CUDART_INF_F;
+    const double a = 1.0 / (double)(1ull << DOM_A), b = 1.0 / (double)(1ull << DOM_B);
+    const bool flat = Z_p > LIST_FLAT_Z && (!nr.hq || Z_q > LIST_FLAT_Z);
+    nr.thrA_p = (float)(Z_p * a);
+    nr.thrB_p = flat ? nr.thrA_p : (float)(Z_p * b);
+    nr.thrA_q = nr.hq ? (float)(Z_q * a) : CUDART_INF_F;
+    nr.thrB_q = nr.hq ? (flat ? nr.thrA_q : (float)(Z_q * b)) : CUDART_INF_F;
 }
 struct RingCtx {
     uint64_t *full, *empty;

@@ -330,6 +330,110 @@ def test_p3_single_path_traversal_is_block_verification_and_beats_naive():
     assert strictly > 0
 
 
+def test_p3_negative_control_literal_reading_of_block_verification_is_not_lossless():
+    """Section 3.1's paragraph read literally -- accept every node independently with probability w_i,
+    return the deepest accepted node, correct from norm((w p - q)+) -- does not reproduce the target
+    law; the enumeration tells the two readings apart (the oracle's reading passes P1 above)."""
+    V, L = 3, 2
+    model = ContextModel(V, L, seed=8)
+    law = {}
+    for xs in itertools.product(range(V), repeat=L):
+        ctx = [tuple(xs[:i]) for i in range(L + 1)]
+        p = [model.p(c) for c in ctx]; q = [model.q(c) for c in ctx]
+        w_path = float(np.prod([q[i][xs[i]] for i in range(L)]))
+        w = [1.0]
+        for i in range(L):
+            w.append(min(1.0, w[i] * p[i][xs[i]] / q[i][xs[i]]))
+        for tau in range(L, -1, -1):
+            # tau = deepest accepted node: node tau accepted (the root always), all deeper ones not
+            pr = (w[tau] if tau > 0 else 1.0) * float(np.prod([1 - w[j] for j in range(tau + 1, L + 1)]))
+            if tau == L:
+                corr = p[L]
+            else:
+                r = np.maximum(w[tau] * p[tau] - q[tau], 0.0)
+                corr = r / r.sum() if r.sum() > 0 else p[tau]
+            for y in range(V):
+                s = tuple(xs[:tau]) + (y,)
+                mass = w_path * pr * corr[y]
+                # continue from p up to length L + 1
+                def ext(s, m):
+                    if len(s) == L + 1:
+                        law[s] = law.get(s, 0.0) + m
+                        return
+                    pn = model.p(s)
+                    for z in range(V):
+                        ext(s + (z,), m * pn[z])
+                ext(s, mass)
+    ref = target_law(model, L + 1)
+    assert abs(sum(law.values()) - 1.0) < 1e-9
+    assert max(abs(law.get(s, 0.0) - ref[s]) for s in ref) > 1e-3
+
+
+def test_traversal_tables_incoming_weights_on_paths_and_leaves():
+    """w_in of oracle.traversal_tables: on a path it is block verification's weight list
+    w_i = min(1, w_{i-1} p(x_i)/q(x_i)) (Section 3.1); at any leaf, reached after its earlier siblings'
+    subtrees were rejected, it is the threshold the leaf is tested with in the enumerated decision
+    tree of the sampling-mode verifier (a leaf's final weight is the weight it was handed)."""
+    V, L = 4, 3
+    rng = np.random.default_rng(61)
+    parent, _ = delayed_tree(1, 0, L)
+    N = L + 1
+    lp = rng.standard_normal((1, N, V)).astype(np.float32) * 1.5
+    lq = rng.standard_normal((1, N, V)).astype(np.float32) * 1.5
+    p, q = softmax64(lp[0]), softmax64(lq[0])
+    for xs in itertools.product(range(V), repeat=L):
+        token = np.array([(0,) + xs], np.int32)
+        w = [1.0]
+        for i in range(L):
+            w.append(min(1.0, w[i] * p[i, xs[i]] / q[i, xs[i]]))
+        w_in, w_fin, _, st = oracle.traversal_tables(tree_inputs(lp, lq, token, np.zeros((1, N), np.float32), parent=parent))
+        np.testing.assert_allclose(w_in[0], w, atol=1e-13)
+        assert w_fin[0, L] == pytest.approx(w[L], abs=1e-13)
+    # branched trees: every leaf's incoming weight against the decision tree of the sampling mode
+    for K, L1, L2, seed in [(3, 0, 1, 1), (2, 1, 1, 2), (2, 0, 2, 3), (3, 1, 1, 4)]:
+        parent, depth = delayed_tree(K, L1, L2)
+        N = len(parent)
+        rng = np.random.default_rng(200 + seed)
+        lp = rng.standard_normal((1, N, V)).astype(np.float32) * 1.2
+        lq = rng.standard_normal((1, N, V)).astype(np.float32) * 1.2
+        token = np.concatenate([[0], rng.integers(0, V, N - 1)]).astype(np.int32)[None]
+        mk = lambda u: tree_inputs(lp, lq, token, u, parent=parent)
+        w_in, w_fin, _, _ = oracle.traversal_tables(mk(np.zeros((1, N), np.float32)))
+        leaves = [a for a in range(1, N) if a not in set(parent[1:].tolist())]
+        seen = {}
+        for prob, node, residual, trace in outcomes(oracle.verify_traversal, mk, N):
+            for tn, thr, _ in trace:
+                seen.setdefault(tn, thr)
+                assert seen[tn] == pytest.approx(thr, abs=1e-13)      # weights do not depend on the decisions
+        for a in leaves:
+            if a in seen:
+                assert w_in[0, a] == pytest.approx(seen[a], abs=1e-13)
+                assert w_fin[0, a] == pytest.approx(seen[a], abs=1e-13)
+        assert any(a in seen for a in leaves)
+        for a in range(1, N):
+            if a in seen:
+                assert w_fin[0, a] == pytest.approx(seen[a], abs=1e-13)
+
+
+def test_traversal_weight_one_is_stable_under_small_residual_masses():
+    """A node of weight exactly 1 keeps weight exactly 1 through every rejected child subtree, however
+    small the residual masses are: w' = S / (S + 1 - w) = 1 (Section 3.1's recursion at w = 1).
+    Four children with the same dominant token in a near-greedy law: S is about 1e-5 at every step."""
+    V = 64
+    rng = np.random.default_rng(4)
+    parent, _ = delayed_tree(4, 0, 1)
+    N = 5
+    base = rng.standard_normal(V).astype(np.float32)
+    base[7] += 12.0                                     # one dominant token in both laws
+    lq = np.repeat(base[None, None], N, 1).astype(np.float32)
+    lp = lq.copy(); lp[0, 0, 7] += 1.5                  # p even more peaked: p(7) > q(7), ratio clipped to 1
+    token = np.array([[0, 7, 7, 7, 7]], np.int32)
+    w_in, w_fin, _, st = oracle.traversal_tables(tree_inputs(lp, lq, token, np.zeros((1, N), np.float32), parent=parent))
+    assert st[0] == 0
+    assert w_fin[0, 0] == 1.0                           # exactly
+    assert w_in[0, 1] == 1.0
+
+
 # ---------------------------------------------------------------------------------------------
 # P4: on a depth-1 tree Traversal and SpecInfer take the same decisions
 # ---------------------------------------------------------------------------------------------
