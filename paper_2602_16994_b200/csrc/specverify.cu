@@ -78,7 +78,8 @@ __global__ void spec_residual_kernel(const RParams P)
 // launch plans
 // ------------------------------------------------------------------------------------------------
 struct VPlan {
-    int C, NW, slice_len, NS, off_x, off_list, off_es, off_ring, smem;
+    int C, NW, slice_len, NS, nsm, off_x, off_list, off_es, off_ring, smem;
+    int whole_sm;       // one CTA per SM: the kernel variant without a register limit may be used
 };
 
 constexpr int SMEM_1CTA = 227 * 1024;          // opt-in limit per CTA
@@ -91,29 +92,34 @@ inline int up(int x, int m) { return (x + m - 1) / m * m; }
 // fits in TMAX tiles of 1792 tokens, fifteen consumer warps (one CTA per SM) above that.
 // Dynamic shared memory: header | exchange slots [2][C][NW][2] doubles | exact lists [NW] | resident e
 // of the tiles that do not fit in registers | ring stages.
-bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bool whole_sm = false)
+bool make_vplan(int V, int dtype, VPlan *p, int hdr_bytes = (int)sizeof(Hdr), bool whole_sm = false, int want_c = 0,
+                int want_nw = 0)
 {
     const int esz = dtype == SPEC_BF16 ? 2 : 4;
     for (int pass = 0; pass < 2; ++pass) {
         const int NW = pass == 0 ? 7 : 15;
+        if (want_nw && NW != want_nw) continue;
         const int tile = NW * 32 * 8;
         const int budget = (NW == 7 && !whole_sm) ? SMEM_2CTA : SMEM_1CTA;
         for (int C = 1; C <= CMAX; C <<= 1) {
+            if (want_c && C != want_c) continue;
             const int slice = up((V + C - 1) / C, 8);
             const int tiles = (slice + tile - 1) / tile;
             if (tiles > TMAX) continue;
-            if (pass == 0 && C > 8) continue;   // prefer one CTA per SM over a non-portable cluster
+            if (pass == 0 && C > 8 && !want_c) continue;   // prefer one CTA per SM over a non-portable cluster
             const int off_x = up(hdr_bytes, 128);
             const int off_list = off_x + up(2 * C * NW * 2 * 8, 128);
             const int off_es = off_list + up(NW * (int)sizeof(WarpList), 128);
-            const int es_bytes = (tiles > RT ? tiles - RT : 0) * tile * 8;
-            const int off_ring = off_es + es_bytes;
             const int stage = 2 * tile * esz;
+            const int nsm = tiles > RT ? tiles - RT : 0;
+            if (nsm > SMT) continue;
+            const int es_bytes = nsm * tile * 8;
+            const int off_ring = off_es + es_bytes;
             int ns = (budget - off_ring) / stage;
             if (ns > NSMAX) ns = NSMAX;
             if (ns > 2 * tiles) ns = 2 * tiles;
             if (ns < 2) continue;
-            p->C = C; p->NW = NW; p->slice_len = slice; p->NS = ns;
+            p->C = C; p->NW = NW; p->slice_len = slice; p->NS = ns; p->nsm = nsm; p->whole_sm = 0;
             p->off_x = off_x; p->off_list = off_list; p->off_es = off_es; p->off_ring = off_ring;
             p->smem = off_ring + ns * stage;
             return true;
@@ -356,10 +362,10 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
 }
 
 // SpecInfer without diagnostic outputs: row statistics of every row, then one walk per sequence
-template <int DT, int NW>
+template <int DT, int NW, int MINB>
 int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
 {
-    auto kernel = spec_walk_kernel<DT, NW>;
+    auto kernel = spec_walk_kernel<DT, NW, MINB>;
     int rc = prepare_kernel(kernel, pl.C, pl.smem);
     if (rc) return rc;
     const int threads = (NW + 1) * 32;
@@ -444,15 +450,16 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
     RowPart *part = (RowPart *)(w + L.stat);
     WParams wp = {};
     wp.B = in->B; wp.N = in->N; wp.V = in->V; wp.C = pl.C; wp.NSL = NSL;
-    wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.off_x = pl.off_x; wp.off_list = pl.off_list; wp.off_es = pl.off_es;
+    wp.slice_len = pl.slice_len; wp.NS = pl.NS; wp.nsm = pl.nsm; wp.off_x = pl.off_x; wp.off_list = pl.off_list; wp.off_es = pl.off_es;
     wp.off_ring = pl.off_ring;
     wp.zp = in->target_logits; wp.zq = in->draft_logits;
     wp.seq_stride = in->seq_stride; wp.node_stride = in->node_stride; wp.topo_stride = in->topo_seq_stride;
     wp.parent = in->parent; wp.token = in->token; wp.T = in->temperature; wp.T_seq = in->temperature_per_seq;
     wp.part = part; wp.u_accept = in->u_accept; wp.u_bonus = in->u_bonus; wp.out = *out;
     const bool bf = in->logits_dtype == SPEC_BF16;
-    if (pl.NW == 7) return bf ? launch_walk<SPEC_BF16, 7>(pl, wp, st) : launch_walk<SPEC_F32, 7>(pl, wp, st);
-    return bf ? launch_walk<SPEC_BF16, 15>(pl, wp, st) : launch_walk<SPEC_F32, 15>(pl, wp, st);
+    if (pl.NW == 7 && pl.whole_sm) return bf ? launch_walk<SPEC_BF16, 7, 1>(pl, wp, st) : launch_walk<SPEC_F32, 7, 1>(pl, wp, st);
+    if (pl.NW == 7) return bf ? launch_walk<SPEC_BF16, 7, 2>(pl, wp, st) : launch_walk<SPEC_F32, 7, 2>(pl, wp, st);
+    return bf ? launch_walk<SPEC_BF16, 15, 1>(pl, wp, st) : launch_walk<SPEC_F32, 15, 1>(pl, wp, st);
 }
 
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode,
@@ -472,12 +479,12 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     const bool diagnostics = out->residual || out->node_thr || out->node_w_in || out->margin;
     if (mode == MODE_SPECINFER && !diagnostics && in->N <= NWALK) {
         // the walk keeps one cluster per sequence busy: when all of them fit on the chip with one CTA
-        // per SM, each CTA may use the whole SM's shared memory for its ring
+        // per SM, each CTA may use the whole SM's shared memory for its ring and twice the registers
         VPlan wpl;
         if (!make_vplan(in->V, in->logits_dtype, &wpl, (int)sizeof(WHdr), false)) return SPEC_ERR_UNSUPPORTED;
         if ((long long)in->B * wpl.C <= sm_count()) {
             VPlan big;
-            if (make_vplan(in->V, in->logits_dtype, &big, (int)sizeof(WHdr), true) && big.C == wpl.C && big.NW == wpl.NW) wpl = big;
+            if (make_vplan(in->V, in->logits_dtype, &big, (int)sizeof(WHdr), true, wpl.C, wpl.NW)) { wpl = big; wpl.whole_sm = 1; }
         }
         return verify_walk(in, out, w, L, wpl, trunc, parts, st);
     }
@@ -489,7 +496,7 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     VParams &vp = tp.v;
     vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
     vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
-    vp.slice_len = pl.slice_len; vp.NS = pl.NS;
+    vp.slice_len = pl.slice_len; vp.NS = pl.NS; vp.nsm = pl.nsm;
     vp.off_x = pl.off_x; vp.off_list = pl.off_list; vp.off_es = pl.off_es; vp.off_ring = pl.off_ring;
     vp.zp = in->target_logits; vp.zq = in->draft_logits;
     vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;

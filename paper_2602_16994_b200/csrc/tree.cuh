@@ -72,7 +72,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     const long long tok0 = (long long)rank * P.slice_len;
     const int n_slice = (int)max(0ll, min((long long)P.slice_len, (long long)P.V - tok0));
     const int ntiles = (n_slice + TILE - 1) / TILE;
-    const int nsm = max(ntiles - RT, 0), nrg = ntiles - nsm;
+    const int nsm = min(P.nsm, ntiles), nrg = ntiles - nsm;
     const bool trav = P.mode == MODE_TRAVERSAL;
 
     if (tid == 0) {

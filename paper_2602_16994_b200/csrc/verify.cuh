@@ -44,8 +44,8 @@
 
 namespace specv {
 
-constexpr int RT = 4;        // tiles per thread whose e live in registers (the kernel names them one by one)
-constexpr int SMT = 6;       // further tiles per thread whose e live in shared memory
+constexpr int RT = 4;        // tiles per thread whose e may live in registers
+constexpr int SMT = 10;      // tiles per thread whose e may live in shared memory
 constexpr int TMAX = RT + SMT;
 constexpr int CMAX = 16;     // CTAs per cluster (above 8: non-portable size)
 constexpr int NSMAX = 16;    // ring stages
@@ -73,6 +73,7 @@ struct VParams {
     int B, N, V, C, mode, all_thr;
     int slice_len;            // tokens per CTA slice: a multiple of 8, at most TMAX tiles
     int NS;                   // ring stages
+    int nsm;                  // tiles of a slice kept in shared memory (the others, at most RT, in registers)
     int off_x, off_list, off_es, off_ring;   // byte offsets inside dynamic shared memory
     const void *zp, *zq;
     long long seq_stride, node_stride, topo_stride;

@@ -29,7 +29,7 @@ constexpr int NWALK = 128;        // nodes per sequence the walk keeps in shared
 
 struct WParams {
     int B, N, V, C, NSL;
-    int slice_len, NS, off_x, off_list, off_es, off_ring;
+    int slice_len, NS, nsm, off_x, off_list, off_es, off_ring;
     const void *zp, *zq;
     long long seq_stride, node_stride, topo_stride;
     const int *parent, *token;
@@ -63,8 +63,9 @@ struct RowSum {
     float cut;
 };
 
-template <int DT, int NW>
-__global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kernel(const WParams P)
+// MINB: CTAs per SM the register budget is set for (1: up to 255 registers per thread, no spills)
+template <int DT, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB) spec_walk_kernel(const WParams P)
 {
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
@@ -83,7 +84,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_walk_kern
     const long long tok0 = (long long)rank * P.slice_len;
     const int n_slice = (int)max(0ll, min((long long)P.slice_len, (long long)P.V - tok0));
     const int ntiles = (n_slice + TILE - 1) / TILE;
-    const int nsm = max(ntiles - RT, 0), nrg = ntiles - nsm;
+    const int nsm = min(P.nsm, ntiles), nrg = ntiles - nsm;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], NW); }
