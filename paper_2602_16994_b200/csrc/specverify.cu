@@ -170,7 +170,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 
 // workspace layout: node records | published weights + arrival counters (cleared per call) | row cuts
 struct WsLayout {
-    int64_t rec, pub, done, cut, todo, stat, gseq, clear_bytes, total;
+    int64_t rec, pub, fin, done, ticket, cut, todo, stat, gseq, total;
 };
 constexpr int MAX_PARTS = 4;      // parts a row may be split into by the streaming statistics kernel
 WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: one record per row only
@@ -179,14 +179,16 @@ WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: on
     const int64_t nodes = (int64_t)in->B * in->N;
     int64_t o = 0;
     L.rec = o; o += up256(nodes * (int64_t)sizeof(NodeRec));
+    // set to all-ones per call: published weights, accepted nodes; set to zero: arrival counters, item counter
     L.pub = o; o += nodes * 8;
+    L.fin = o; o += (int64_t)in->B * 4;
     L.done = o; o += (int64_t)in->B * 4;
-    L.clear_bytes = o - L.pub;
+    L.ticket = o; o += 4;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
     L.todo = o; o += up256(4 + nodes * 8);          // count, then ids of the rows left to the general top-k / top-p kernel
     L.stat = o; o += up256(nodes * 2 * (slices + 1) * (int64_t)sizeof(RowPart));      // one record per row, then the parts
-    L.gseq = o; o += up256(nodes * KMAX * 8);       // step coefficients of every node (written only for the residual output)
+    L.gseq = o; o += up256(nodes * KMAX * 8);       // step coefficients of every node
     L.total = o;
     return L;
 }
@@ -302,8 +304,8 @@ int launch_tree(const VPlan &pl, TParams &tp, cudaStream_t st)
     const int threads = (NW + 1) * 32;
     int nc = resident_clusters(kernel, pl.C, threads, pl.smem);
     if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
-    const long long nodes = (long long)tp.v.B * tp.v.N;
-    if (nc > nodes) nc = (int)nodes;
+    const long long items = (long long)tp.v.B * tp.v.N + tp.v.B;
+    if (nc > items) nc = (int)items;
     return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &tp);
 }
 
@@ -386,8 +388,8 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
     RowPart *part = (RowPart *)(w + L.stat);
     if (trunc) {
         if (init_nodes &&
-            (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)((int64_t)in->B * in->N * 8), st) != cudaSuccess ||
-             cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4, st) != cudaSuccess)) {
+            (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)(L.done - L.pub), st) != cudaSuccess ||
+             cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4 + 4, st) != cudaSuccess)) {
             cudaGetLastError();
             return SPEC_ERR_CUDA;
         }
@@ -408,7 +410,10 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
         // in one part is final as written.  One CTA per item: those of unread rows retire at once.
         RowPart *parts = part + 2ll * in->B * in->N;
         sp.part = NSL > 1 ? parts : part;
-        if (init_nodes) { sp.w_pub = (unsigned long long *)(w + L.pub); sp.done = (unsigned int *)(w + L.done); }
+        if (init_nodes) {
+            sp.w_pub = (unsigned long long *)(w + L.pub); sp.done = (unsigned int *)(w + L.done);
+            sp.fin = (int *)(w + L.fin); sp.ticket = (unsigned int *)(w + L.ticket);
+        }
         const long long items = 2ll * in->B * in->N * NSL;
         const unsigned grid = (unsigned)(items < (1ll << 20) ? items : (1ll << 20));
         int prc;
@@ -506,9 +511,11 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     vp.rec = (NodeRec *)(w + L.rec);
     vp.w_pub = (unsigned long long *)(w + L.pub);
     vp.done = (unsigned int *)(w + L.done);
+    vp.fin = (int *)(w + L.fin);
     vp.out = *out;
     tp.part = (const RowPart *)(w + L.stat);
-    tp.gseq = out->residual ? (double *)(w + L.gseq) : nullptr;
+    tp.gseq = (double *)(w + L.gseq);
+    tp.ticket = (unsigned int *)(w + L.ticket);
     const bool bf = in->logits_dtype == SPEC_BF16;
     if (pl.NW == 7) rc = bf ? launch_tree<SPEC_BF16, 7>(pl, tp, st) : launch_tree<SPEC_F32, 7>(pl, tp, st);
     else rc = bf ? launch_tree<SPEC_BF16, 15>(pl, tp, st) : launch_tree<SPEC_F32, 15>(pl, tp, st);

@@ -37,10 +37,13 @@ struct SParams {
     float T;
     const float *T_seq;
     RowPart *part;           // [B*N*2][NSL]
-    // optional (every-node verification follows): the per-node weight slots are set to pending and the
-    // per-sequence arrival counters to zero here, which saves two memset nodes per call
+    // optional (every-node verification follows): the per-node weight slots and the per-sequence accepted-node
+    // slots are set to pending, the arrival counters and the item counter to zero here, which saves the memset
+    // nodes of a call
     unsigned long long *w_pub;   // [B*N]
     unsigned int *done;          // [B]
+    int *fin;                    // [B] set to -1 (no accepted node selected yet)
+    unsigned int *ticket;        // [1] item counter of the every-node kernel
 };
 
 // depth of the per-thread staging ring and its size
@@ -96,7 +99,8 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         RowPart *out = P.part + row2 * P.NSL + h;
         if (P.w_pub && which == 0 && h == 0 && tid == 0) {
             P.w_pub[row] = W_PENDING;
-            if (a == 0) P.done[b] = 0u;
+            if (a == 0) { P.done[b] = 0u; P.fin[b] = -1; }
+            if (row == 0) *P.ticket = 0u;
         }
         if (which == 1) {
             // a draft row is read only for nodes that have children (every warp finds out by itself)

@@ -3,10 +3,17 @@
 // weights are defined for every node, top-down: Section 3.2) and as SpecInfer's diagnostic outputs
 // need (the threshold of every node, Algorithm 4).
 //
+// Items are handed out at run time: the producer warp of a cluster's first CTA draws a ticket from a
+// counter in the workspace and passes it to the other CTAs' producers through distributed shared
+// memory.  Tickets 0 .. B N - 1 are the nodes in node-major order (parents first), tickets B N ..
+// B N + B - 1 one FINISH item per sequence.  A node waits only for the weight its parent publishes,
+// the parent holds a smaller ticket, and a ticket is drawn only by a running cluster, so the smallest
+// unfinished ticket never waits on anything unfinished -- whatever share of the grid is resident.
+//
 // With a row's reference O and normaliser Z known before the node comes on chip, a node is:
 //   scalars   children, their tokens and uniforms, the exact exponentials 2^(z s - O) of every child's
-//             token in both rows -- gathered by the producer warp, one node ahead of the consumers,
-//             into a double-buffered block of shared memory;
+//             token in both rows -- gathered by the producer warp, ahead of the consumers, into a
+//             double-buffered block of shared memory;
 //   pass 1    e = 2^(z s - O) of both rows, resident in registers and shared memory, all threads in
 //             the same units; the dominant tokens in fp64 on the warps' exact lists (verify.cuh);
 //   Z         the rows' normalisers again, from the resident e and the lists (one exchange): the
@@ -15,10 +22,14 @@
 //   siblings  the residual recursion of verify.cuh, step by step: u <- (g u - e_q)+ in place, one sweep
 //             over the resident data and one distributed-shared-memory exchange per rejected child;
 //             child j is handed min(1, w P(x_j) / q(x_j)) from the state before its step, published at once;
-//   outcome   the node's final weight; where the node can be the accepted one, the bonus token by an
-//             inverse-CDF search over the final state.
-// Records, published weights, arrival counting and the writing of a sequence's outputs are those of
-// verify.cuh.
+//   outcome   the node's final weight and the coefficients g_j of its steps, recorded.
+// A childless node needs no rows and no item of its own: its weight is the one it is handed, so the
+// parent's scribe warp writes its record and makes its arrival when it publishes that weight (its ticket
+// is skipped by every producer).  A node whose weight is already known to be 0 when its ticket is drawn
+// needs no rows either (nothing below it can be accepted).
+// The warp that makes the last of a sequence's arrivals selects the accepted node and publishes it;
+// the sequence's FINISH item brings that one node back on chip, replays its recorded steps (no
+// exchange: the coefficients are known) and draws the bonus token by the inverse-CDF search.
 #pragma once
 #include "stream.cuh"
 #include "verify.cuh"
@@ -28,27 +39,66 @@ namespace specv {
 struct TParams {
     VParams v;                // shapes, inputs, records, published weights, arrival counters, outputs
     const RowPart *part;      // [B*N*2] statistics of every row the verifier reads
-    double *gseq;             // optional [B*N][KMAX]: the step coefficients g_j of every node (for the residual output)
+    double *gseq;             // [B*N][KMAX]: the step coefficients g_j of every node
+    unsigned int *ticket;     // item counter (0 at launch)
 };
 
-// what the consumers need to know about a node besides its rows
+// ITEM_LEAF: a childless root (a tree of one node); other childless nodes are never items
+enum ItemKind { ITEM_NODE = 0, ITEM_LEAF = 1, ITEM_DEAD = 2, ITEM_FINISH = 3, ITEM_IDLE = 4, ITEM_EXIT = 5 };
+
+// what the consumers need to know about an item besides its rows
 struct __align__(16) NodeScalars {
     double Z_p, Z_q;
-    double cpm[KMAX], cqm[KMAX];   // exact 2^(z s - O) of the children's tokens in the node's target and draft rows
+    double cpm[KMAX], cqm[KMAX];   // node: exact 2^(z s - O) of the children's tokens in the node's target and draft
+                                   // rows; FINISH item: cpm = the recorded coefficients g_j
     float cu[KMAX];                // the children's acceptance uniforms
     int child[KMAX];
     int kc, err, O_p, O_q;
     float cut_p, cut_q, u_a, ub_a;
+    int kind, a, b, nsteps;
+    unsigned leaf_mask;            // bit j: child j has no children
+    int pad[3];
 };
 
 struct __align__(16) THdr {
-    uint64_t full[NSMAX], empty[NSMAX], xbar[2], cbar, sfull[2], sempty[2];
+    uint64_t full[NSMAX], empty[NSMAX], xbar[2], cbar, sfull[2], sempty[2], tbar[2], abar[2];
+    unsigned long long item[2];    // ticket | (weight already 0) << 32, written by the first CTA's producer
     double wtile[NWMAX + 1][TMAX];
     NodeScalars sc[2];
     int poison;
 };
 
 static_assert(sizeof(THdr) <= sizeof(Hdr), "the launch plan reserves sizeof(Hdr) bytes for the header");
+
+__device__ __forceinline__ void st_async_u64(unsigned long long *slot, uint64_t *bar, uint32_t rank, unsigned long long v)
+{
+    asm volatile(
+        "{\n\t.reg .b32 ra, rb;\n\tmapa.shared::cluster.u32 ra, %0, %2;\n\tmapa.shared::cluster.u32 rb, %1, %2;\n\t"
+        "st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [ra], %3, [rb];\n\t}" ::"r"(smem_u32(slot)),
+        "r"(smem_u32(bar)), "r"(rank), "l"(v)
+        : "memory");
+}
+// one arrival on the mbarrier at the same offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint64_t *bar, uint32_t rank)
+{
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(smem_u32(bar)), "r"(rank)
+        : "memory");
+}
+// bounded poll of a published weight; W_PENDING when the limit ran out
+__device__ __forceinline__ unsigned long long poll_weight(const unsigned long long *slot_, const int *poison)
+{
+    volatile const unsigned long long *slot = slot_;
+    const long long t0 = clock64();
+    unsigned long long bits;
+    for (;;) {
+        bits = *slot;
+        if (bits != W_PENDING || clock64() - t0 > WAIT_CYCLES || *(volatile const int *)poison) break;
+        __nanosleep(32);
+    }
+    return bits;
+}
 
 template <int DT, int NW>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kernel(const TParams TP)
@@ -67,7 +117,6 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     unsigned char *ring = dyn_smem + P.off_ring;
     const int C = P.C, NS = P.NS;
     const unsigned rank = cluster_ctarank();
-    const int cid = blockIdx.x / C, NC = gridDim.x / C;
     const long long total = (long long)P.B * P.N;
     const long long tok0 = (long long)rank * P.slice_len;
     const int n_slice = (int)max(0ll, min((long long)P.slice_len, (long long)P.V - tok0));
@@ -79,10 +128,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         for (int s = 0; s < NS; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], NW); }
         mbar_init(&S.xbar[0], 1);
         mbar_init(&S.xbar[1], 1);
-        mbar_init(&S.sfull[0], 1);
-        mbar_init(&S.sfull[1], 1);
-        mbar_init(&S.sempty[0], NW);
-        mbar_init(&S.sempty[1], NW);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&S.sfull[i], 1);
+            mbar_init(&S.sempty[i], NW);
+            mbar_init(&S.tbar[i], 1);
+            mbar_init(&S.abar[i], C);
+        }
         mbar_init(&S.cbar, NW);
         S.poison = 0;
         mbar_fence_init();
@@ -91,100 +142,197 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
     cluster_sync_all();
 
     if (warp == NW) {
-        // ======================= producer warp: fills the ring, node after node, and gathers the =======
-        // ======================= scalars of the node after the one whose rows it has just issued =======
-        int g = 0;
+        // ======================= producer warp: draws items, gathers their scalars, fills the ring ==============
+        int g = 0, sidx = 0;          // ring uses so far; scalars blocks handed to the consumers so far
         bool ok = true;
-        // scalars of item `id` (the kidx-th item of this cluster) into block kidx & 1
-        auto scalars = [&](long long id, int kidx) {
-            const int a = (int)(id / P.B), b = (int)(id % P.B);
+        for (int kidx = 0; ok; ++kidx) {
             const int buf = kidx & 1;
-            if (kidx >= 2) {
+            // ---- the item: drawn by the first CTA's producer, passed on to the others ---------------------------
+            if (rank == 0) {
+                unsigned long long val = 0;
                 int w = 1;
-                if (lane == 0) w = mbar_wait(&S.sempty[buf], (uint32_t)(((kidx >> 1) - 1) & 1)) ? 1 : 0;
-                w = __shfl_sync(0xffffffffu, w, 0);
-                if (!w || *(volatile int *)&S.poison) { S.poison = 1; ok = false; return; }
-            }
-            NodeScalars &N = S.sc[buf];
-            const int *parent = P.parent + (long long)b * P.topo_stride;
-            const int *token = P.token + (long long)b * P.N;
-            const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-            int kc = 0, err = 0;
-            if (lane == 0) {
-                const int pa = __ldg(parent + a);
-                if (a == 0 ? (pa != -1) : (pa < 0 || pa >= a)) err = SPEC_DEV_TOPOLOGY;
-                if (a > 0) {
-                    const int x = __ldg(token + a);
-                    if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                if (lane == 0) {
+                    // every producer has read the item that used this slot before
+                    if (kidx >= 2) w = mbar_wait_cluster(&S.abar[buf], (uint32_t)(((kidx >> 1) - 1) & 1)) ? 1 : 0;
+                    const unsigned t = atomicAdd(TP.ticket, 1u);
+                    unsigned hint = 0;
+                    if (trav && (long long)t < total && t >= (unsigned)P.B) {
+                        // a node whose weight is already known to be 0 needs no rows
+                        const int a = (int)(t / (unsigned)P.B), b = (int)(t % (unsigned)P.B);
+                        if (*(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + a) == 0ull) hint = 1;
+                    }
+                    val = (unsigned long long)t | ((unsigned long long)hint << 32);
                 }
-                N.u_a = __ldg(P.u_accept + (long long)b * P.N + a);
-                N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
+                w = __shfl_sync(0xffffffffu, w, 0);
+                val = __shfl_sync(0xffffffffu, val, 0);
+                if (!w) { S.poison = 1; val = 0xFFFFFFFFull; }       // gave up: everybody leaves
+                if (lane < C) st_async_u64(&S.item[buf], &S.tbar[buf], (uint32_t)lane, val);
             }
-            int my_tok = 0;              // lanes j and 16 + j: token of child j
-            for (int c0 = a + 1; c0 < P.N; c0 += 32) {
-                const int c = c0 + lane;
-                const bool is = c < P.N && __ldg(parent + c) == a;
-                const unsigned bal = __ballot_sync(0xffffffffu, is);
-                if (is) {
-                    const int pos = kc + __popc(bal & ((1u << lane) - 1u));
-                    if (pos < KMAX) {
-                        const int x = __ldg(token + c);
-                        N.child[pos] = c;
-                        N.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
-                        N.cpm[pos] = (double)x;          // parked here until the probabilities are known
+            unsigned long long item = 0;
+            {
+                int w = 1;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&S.tbar[buf], 8u);
+                    w = mbar_wait_cluster(&S.tbar[buf], (uint32_t)((kidx >> 1) & 1)) ? 1 : 0;
+                    item = *(volatile unsigned long long *)&S.item[buf];
+                    mbar_arrive_remote(&S.abar[buf], 0u);
+                }
+                w = __shfl_sync(0xffffffffu, w, 0);
+                item = __shfl_sync(0xffffffffu, item, 0);
+                if (!w) { S.poison = 1; item = 0xFFFFFFFFull; }
+            }
+            const long long t = (long long)(item & 0xFFFFFFFFull);
+            const bool hint_dead = (item >> 32) != 0;
+
+            // a childless node other than the root is finished by its parent: its ticket is skipped by everybody
+            // (one whose parent index is not valid is nobody's child: it stays an item and reports the fault)
+            if (t >= P.B && t < total) {
+                const int a_ = (int)(t / P.B), b_ = (int)(t % P.B);
+                const int *par_ = P.parent + (long long)b_ * P.topo_stride;
+                const int pa_ = __ldg(par_ + a_);
+                if (pa_ >= 0 && pa_ < a_ && !warp_has_children(par_, P.N, a_, lane)) continue;
+            }
+
+            // ---- the scalars block of this item -----------------------------------------------------------------
+            const int sbuf = sidx & 1;
+            if (sidx >= 2) {
+                int w = 1;
+                if (lane == 0) w = mbar_wait(&S.sempty[sbuf], (uint32_t)(((sidx >> 1) - 1) & 1)) ? 1 : 0;
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (!w) S.poison = 1;
+            }
+            ++sidx;
+            NodeScalars &N = S.sc[sbuf];
+            int kind, a = 0, b = 0;
+            bool hq = false;
+            if (t >= total + P.B || *(volatile int *)&S.poison) {
+                kind = ITEM_EXIT;
+                ok = false;
+            } else if (t >= total) {
+                // FINISH: wait (bounded) until the sequence's accepted node is published
+                kind = ITEM_FINISH;
+                b = (int)(t - total);
+                int acc = FIN_PENDING;
+                if (lane == 0) {
+                    volatile int *slot = P.fin + b;
+                    const long long t0 = clock64();
+                    for (;;) {
+                        acc = *slot;
+                        if (acc != FIN_PENDING || clock64() - t0 > WAIT_CYCLES || *(volatile int *)&S.poison) break;
+                        __nanosleep(64);
+                    }
+                    __threadfence();       // the records written before the publication are read below
+                }
+                acc = __shfl_sync(0xffffffffu, acc, 0);
+                int err = 0;
+                if (acc == FIN_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; }
+                if (acc < 0 || err) {
+                    kind = ITEM_IDLE;           // a faulty sequence has no bonus draw
+                    if (lane == 0) { N.err = err; N.b = b; N.a = -1; }
+                } else {
+                    a = acc;
+                    const NodeRec *rc = P.rec + (long long)b * P.N + a;
+                    const int nsteps = __ldcg(&rc->nsteps);
+                    hq = nsteps != 0;
+                    if (lane < KMAX && lane < nsteps) N.cpm[lane] = __ldcg(TP.gseq + ((long long)b * P.N + a) * KMAX + lane);
+                    if (lane == 0) {
+                        N.Z_p = __ldcg(&rc->Z_p); N.Z_q = __ldcg(&rc->Z_q);
+                        N.O_p = (int)__ldcg(&rc->O_p); N.O_q = (int)__ldcg(&rc->O_q);
+                        N.cut_p = __ldcg(&rc->cut_p); N.cut_q = __ldcg(&rc->cut_q);
+                        N.nsteps = nsteps; N.kc = hq ? 1 : 0; N.err = 0; N.a = a; N.b = b;
+                        N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
+                    }
+                }
+            } else {
+                a = (int)(t / P.B);
+                b = (int)(t % P.B);
+                const int *parent = P.parent + (long long)b * P.topo_stride;
+                const int *token = P.token + (long long)b * P.N;
+                const double s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+                int kc = 0, err = 0;
+                if (lane == 0) {
+                    const int pa = __ldg(parent + a);
+                    if (a == 0 ? (pa != -1) : (pa < 0 || pa >= a)) err = SPEC_DEV_TOPOLOGY;
+                    if (a > 0) {
+                        const int x = __ldg(token + a);
                         if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
                     }
+                    N.u_a = __ldg(P.u_accept + (long long)b * P.N + a);
+                    N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
+                    N.a = a; N.b = b; N.nsteps = 0;
                 }
-                kc += __popc(bal);
-            }
-            if (kc > KMAX) err = SPEC_DEV_TOPOLOGY;
-            const bool hq = kc > 0;
-            const RowPart *rp = TP.part + ((long long)b * P.N + a) * 2;
-            const double Z_p = __ldcg(&rp[0].S);
-            const int O_p = __ldcg(&rp[0].O);
-            const float cut_p = __ldcg(&rp[0].cut);
-            double Z_q = 0.0;
-            int O_q = ROWPART_EMPTY;
-            float cut_q = -CUDART_INF_F;
-            bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
-            if (hq) {
-                Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
-                bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
-            }
-            err = __reduce_max_sync(0xffffffffu, err);
-            if (bad && !err) err = SPEC_DEV_NONFINITE;
-            __syncwarp();
-            {
-                const int j = lane & 15;
-                const bool mine = !err && j < kc;
-                my_tok = mine ? (int)N.cpm[j] : 0;
-                __syncwarp();
-                double pr = 0.0;
-                if (mine) {
-                    const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
-                    const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + my_tok);
-                    const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
-                    if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
-                        const double nd = rint(xd);
-                        pr = exp2_frac_once(xd - nd) * pow2d((int)nd);
+                for (int c0 = a + 1; c0 < P.N; c0 += 32) {
+                    const int c = c0 + lane;
+                    const bool is = c < P.N && __ldg(parent + c) == a;
+                    const unsigned bal = __ballot_sync(0xffffffffu, is);
+                    if (is) {
+                        const int pos = kc + __popc(bal & ((1u << lane) - 1u));
+                        if (pos < KMAX) {
+                            const int x = __ldg(token + c);
+                            N.child[pos] = c;
+                            N.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
+                            N.cpm[pos] = (double)x;          // parked here until the exponentials are known
+                            if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
+                        }
                     }
+                    kc += __popc(bal);
                 }
-                if (j < KMAX) { if (lane < 16) N.cpm[j] = pr; else N.cqm[j] = pr; }
+                if (kc > KMAX) err = SPEC_DEV_TOPOLOGY;
+                hq = kc > 0;
+                // which children are childless (their grandchildren name them as parent)
+                unsigned nonleaf = 0;
+                __syncwarp();
+                for (int d0 = a + 2; d0 < P.N; d0 += 32) {
+                    const int d = d0 + lane;
+                    const int pd = d < P.N ? __ldg(parent + d) : -1;
+                    for (int j = 0; j < min(kc, KMAX); ++j)
+                        if (pd == N.child[j]) nonleaf |= 1u << j;
+                }
+                nonleaf = __reduce_or_sync(0xffffffffu, nonleaf);
+                const RowPart *rp = TP.part + ((long long)b * P.N + a) * 2;
+                const double Z_p = __ldcg(&rp[0].S);
+                const int O_p = __ldcg(&rp[0].O);
+                const float cut_p = __ldcg(&rp[0].cut);
+                double Z_q = 0.0;
+                int O_q = ROWPART_EMPTY;
+                float cut_q = -CUDART_INF_F;
+                bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
+                if (hq) {
+                    Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
+                    bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
+                }
+                err = __reduce_max_sync(0xffffffffu, err);
+                if (bad && !err) err = SPEC_DEV_NONFINITE;
+                kind = (hint_dead || err) ? ITEM_DEAD : (hq ? ITEM_NODE : ITEM_LEAF);
+                __syncwarp();
+                if (kind == ITEM_NODE) {
+                    const int j = lane & 15;
+                    const bool mine = j < kc;
+                    const int my_tok = mine ? (int)N.cpm[j] : 0;
+                    __syncwarp();
+                    double pr = 0.0;
+                    if (mine) {
+                        const long long rowb = (long long)b * P.seq_stride + (long long)a * P.node_stride;
+                        const float z = load_logit(lane < 16 ? P.zp : P.zq, DT, rowb + my_tok);
+                        const double xd = (double)z * s_d - (double)(lane < 16 ? O_p : O_q);
+                        if (z >= (lane < 16 ? cut_p : cut_q) && xd > -1000.0) {
+                            const double nd = rint(xd);
+                            pr = exp2_frac_once(xd - nd) * pow2d((int)nd);
+                        }
+                    }
+                    if (j < KMAX) { if (lane < 16) N.cpm[j] = pr; else N.cqm[j] = pr; }
+                }
+                if (lane == 0) {
+                    N.Z_p = Z_p; N.Z_q = Z_q; N.O_p = O_p; N.O_q = O_q; N.cut_p = cut_p; N.cut_q = cut_q;
+                    N.kc = kc; N.err = err; N.leaf_mask = ~nonleaf;
+                }
             }
-            if (lane == 0) {
-                N.Z_p = Z_p; N.Z_q = Z_q; N.O_p = O_p; N.O_q = O_q; N.cut_p = cut_p; N.cut_q = cut_q;
-                N.kc = kc; N.err = err;
-            }
+            if (lane == 0) N.kind = kind;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S.sfull[buf]);
-        };
-        // pass 1 needs a node's references and cuts, so its scalars come before its rows: the first
-        // node's before anything else, from then on one node ahead
-        int kidx = 0;
-        if (cid < total) scalars(cid, 0);
-        for (long long id = cid; id < total && ok; id += NC, ++kidx) {
-            const int a = (int)(id / P.B), b = (int)(id % P.B);
-            const bool hq = warp_has_children(P.parent + (long long)b * P.topo_stride, P.N, a, lane);
+            if (lane == 0) mbar_arrive(&S.sfull[sbuf]);
+            if (kind != ITEM_NODE && kind != ITEM_FINISH) continue;
+
+            // ---- the item's rows through the ring -------------------------------------------------------------------
             const long long row = (long long)b * P.seq_stride + (long long)a * P.node_stride + tok0;
             const unsigned char *src_p = (const unsigned char *)P.zp + row * ESZ;
             const unsigned char *src_q = (const unsigned char *)P.zq + row * ESZ;
@@ -224,10 +372,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     }
                 }
             }
-            if (!ok) break;
-            if (id + NC < total) scalars(id + NC, kidx + 1);
         }
-        if (!ok && lane == 0) {
+        if (*(volatile int *)&S.poison && lane == 0) {
             // gave up: wait (bounded) for the copies still in flight before leaving
             for (int k = 1; k <= NS && k <= g; ++k) {
                 const int gg = g - k;
@@ -242,203 +388,298 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         int stage = 0;
         uint32_t phase = 0, cph = 0;
         int xn = 0;
-        int kidx = 0;
         Resident R;
 
-        for (long long id = cid; id < total; id += NC, ++kidx) {
-            const int a = (int)(id / P.B), b = (int)(id % P.B);
-            const int *parent = P.parent + (long long)b * P.topo_stride;
-            NodeRows nr;
-            nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-            nr.s_hi = (float)nr.s_d;
-            if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
-            nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
-            if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
-
-            // ---- the node's scalars, gathered by the producer warp --------------------------------------------
+        for (int kidx = 0;; ++kidx) {
+            // ---- the item's scalars, gathered by the producer warp ------------------------------------------------
             bool poisoned = *(volatile int *)&S.poison != 0;
             const NodeScalars &W = S.sc[kidx & 1];
             if (!poisoned && !mbar_wait(&S.sfull[kidx & 1], (uint32_t)((kidx >> 1) & 1))) { S.poison = 1; poisoned = true; }
-            int err = poisoned ? SPEC_DEV_TIMEOUT : W.err;
-            const int kc = poisoned ? 0 : W.kc;
-            const bool hq = kc > 0;
-            nr.hq = hq; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
-            set_list_thresholds(nr, W.Z_p, W.Z_q);
+            const int kind = poisoned ? ITEM_EXIT : W.kind;
+            if (kind == ITEM_EXIT) break;
+            const int a = W.a, b = W.b;
+            int err = W.err;
+            const int *parent = P.parent + (long long)b * P.topo_stride;
 
-            // ---- pass 1: e = 2^(z s - O) of both rows, resident; dominant tokens to the exact lists -------------
-            int nl;
-            float zs_p, zs_q;
-            pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
-            if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
-
-            // ---- the rows' normalisers from what is resident (one exchange; a childless node needs none:
-            // its weight is its parent's, and the bonus search works on unnormalised totals) -----------------
-            double Z_p = W.Z_p, Z_q = W.Z_q;
-            double Zr_p = 0.0, Zr_q = 0.0;        // lane r: rank r's share of the normalisers
-            if (hq && !err) {
-                const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
-                                     warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
-                double tot[2], mine[2];
-                cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                if (*(volatile int *)&S.poison) err = SPEC_DEV_TIMEOUT;
-                else if (!(tot[0] > 0.0) || !(tot[1] > 0.0)) err = SPEC_DEV_NONFINITE;
-                else { Z_p = tot[0]; Z_q = tot[1]; Zr_p = mine[0]; Zr_q = mine[1]; }
-            }
-            const double invZq = (err || !hq) ? 0.0 : __drcp_rn(Z_q);
-
-            // ---- Traversal: the weight handed down by the parent (bounded poll, every warp for itself) ------
-            double w_in = 1.0;
-            if (trav && a > 0 && !err) {
-                unsigned long long bits = W_PENDING;
+            // a childless child is finished here, by the scribe warp: its record and its arrival
+            auto finish_leaf = [&](int c, double thr_c) {
                 if (lane == 0) {
-                    volatile unsigned long long *slot = P.w_pub + (long long)b * P.N + a;
-                    const long long t0 = clock64();
-                    for (;;) {
-                        bits = *slot;
-                        if (bits != W_PENDING || clock64() - t0 > WAIT_CYCLES || *(volatile int *)&S.poison) break;
-                        __nanosleep(32);
-                    }
+                    NodeRec &Rl = P.rec[(long long)b * P.N + c];
+                    const RowPart *rpl = TP.part + ((long long)b * P.N + c) * 2;
+                    const double Zl = __ldcg(&rpl->S);
+                    const int Ol = __ldcg(&rpl->O);
+                    const bool badl = __ldcg(&rpl->bad) != 0 || !(Ol > ROWPART_EMPTY) || !(Zl > 0.0) || !(Zl < CUDART_INF);
+                    Rl.O_p = (double)Ol; Rl.Z_p = Zl; Rl.O_q = 0.0; Rl.Z_q = 0.0;
+                    Rl.kappa = Zl; Rl.nsteps = 0;
+                    Rl.cut_p = __ldcg(&rpl->cut); Rl.cut_q = -CUDART_INF_F;
+                    Rl.next_child = -1;
+                    Rl.status = badl ? SPEC_DEV_NONFINITE : 0;
+                    Rl.bonus = -1; Rl.bonus_margin = 0.f;
+                    Rl.w_in = trav ? thr_c : 1.0;
+                    Rl.thr = thr_c;
                 }
-                bits = __shfl_sync(0xffffffffu, bits, 0);
-                if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
-                else w_in = __longlong_as_double((long long)bits);
-            }
+                arrive_sequence(P, b);
+            };
 
-            // ---- the recursion, step by step (identical in every warp of the cluster) ---------------------------
-            // state: the resident u (total kappa), the node's weight w, and in lane j < kc the value of u at
-            // child j's token with its e_q (fp64, the same recursion as the vocabulary)
-            const bool live = !err && w_in > 0.0;
-            double w = live ? w_in : 0.0, kappa = Z_p;
-            bool dead = !live, is_q = false;      // is_q: a step with S = 0 at weight 1 showed that the state equals q
-            int nsteps = 0;
-            const int kce = min(kc, KMAX);
-            double ux = (lane < kce) ? W.cpm[lane] : 0.0;
-            const double eqx = (lane < kce) ? W.cqm[lane] : 0.0;
-            double tot_r = hq ? Zr_p : 0.0;       // lane r: rank r's share of kappa (childless node: exchanged below)
-            double *gs = TP.gseq ? TP.gseq + ((long long)b * P.N + a) * KMAX : nullptr;
-            int acc = -1;
-            if (err && scribe && lane == 0) {
-                // nothing below a faulty node is evaluated: every child gets weight / threshold 0
-                NodeRec *rec = P.rec + (long long)b * P.N;
-                for (int c = a + 1; c < P.N; ++c)
-                    if (__ldg(parent + c) == a) {
-                        if (trav) {
-                            rec[c].w_in = 0.0;
-                            *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
-                        } else {
-                            rec[c].thr = 0.0;
+            if (kind == ITEM_IDLE) {
+                // a sequence without a bonus draw: its status says why (a timeout met here is added)
+                if (scribe && lane == 0 && err) P.out.status[b] = err;
+            } else if (kind == ITEM_LEAF || kind == ITEM_DEAD) {
+                // ---- no rows: a childless node is tested with the weight it was handed; nothing under a node of
+                // weight 0 (or under a faulty node) can be accepted -----------------------------------------------
+                if (scribe) {
+                    double w_in = 1.0;
+                    if (trav && a > 0 && !err) {
+                        unsigned long long bits = W_PENDING;
+                        if (lane == 0) bits = poll_weight(P.w_pub + (long long)b * P.N + a, &S.poison);
+                        bits = __shfl_sync(0xffffffffu, bits, 0);
+                        if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
+                        else w_in = __longlong_as_double((long long)bits);
+                    }
+                    if (lane == 0) {
+                        NodeRec *rec = P.rec + (long long)b * P.N;
+                        NodeRec &Rc = rec[a];
+                        Rc.O_p = (double)W.O_p; Rc.Z_p = W.Z_p; Rc.O_q = (double)W.O_q; Rc.Z_q = W.Z_q;
+                        Rc.kappa = W.Z_p; Rc.nsteps = 0;
+                        Rc.cut_p = W.cut_p; Rc.cut_q = W.cut_q;
+                        Rc.next_child = -1;
+                        Rc.status = err;
+                        Rc.bonus = -1; Rc.bonus_margin = 0.f;
+                        if (trav) { Rc.thr = (a == 0) ? 1.0 : (err ? 0.0 : w_in); if (a == 0) Rc.w_in = 1.0; }
+                        else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
+                    }
+                    // the children of a node of weight 0 (or of a faulty one) get weight / threshold 0 at once
+                    if (kind == ITEM_DEAD && W.kc > KMAX) {
+                        // too many children to list: found by scanning
+                        for (int c = a + 1; c < P.N; ++c) {
+                            if (__ldg(parent + c) != a) continue;
+                            if (!warp_has_children(parent, P.N, c, lane)) { finish_leaf(c, 0.0); continue; }
+                            if (lane == 0) {
+                                NodeRec *rec = P.rec + (long long)b * P.N;
+                                if (trav) {
+                                    rec[c].w_in = 0.0;
+                                    *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
+                                } else {
+                                    rec[c].thr = 0.0;
+                                }
+                            }
+                        }
+                    } else if (kind == ITEM_DEAD)
+                        for (int j = 0; j < W.kc; ++j) {
+                            const int c = W.child[j];
+                            if ((W.leaf_mask >> j) & 1u) { finish_leaf(c, 0.0); continue; }
+                            if (lane == 0) {
+                                NodeRec *rec = P.rec + (long long)b * P.N;
+                                if (trav) {
+                                    rec[c].w_in = 0.0;
+                                    *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
+                                } else {
+                                    rec[c].thr = 0.0;
+                                }
+                            }
+                        }
+                    arrive_sequence(P, b);
+                }
+            } else if (kind == ITEM_NODE) {
+                NodeRows nr;
+                nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+                nr.s_hi = (float)nr.s_d;
+                if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
+                nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
+                if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
+                const int kc = W.kc;
+                nr.hq = true; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
+                set_list_thresholds(nr, W.Z_p, W.Z_q);
+
+                // ---- pass 1: e = 2^(z s - O) of both rows, resident; dominant tokens to the exact lists -------------
+                int nl;
+                float zs_p, zs_q;
+                pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
+                if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
+
+                // ---- the rows' normalisers from what is resident (one exchange) -----------------------------------
+                double Z_p = W.Z_p, Z_q = W.Z_q;
+                {
+                    const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
+                                         warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
+                    double tot[2], mine[2];
+                    cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                    if (*(volatile int *)&S.poison) err = SPEC_DEV_TIMEOUT;
+                    else if (!(tot[0] > 0.0) || !(tot[1] > 0.0)) err = SPEC_DEV_NONFINITE;
+                    else { Z_p = tot[0]; Z_q = tot[1]; }
+                }
+                const double invZq = err ? 0.0 : __drcp_rn(Z_q);
+
+                // ---- Traversal: the weight handed down by the parent (bounded poll, every warp for itself) ------
+                double w_in = 1.0;
+                if (trav && a > 0 && !err) {
+                    unsigned long long bits = W_PENDING;
+                    if (lane == 0) bits = poll_weight(P.w_pub + (long long)b * P.N + a, &S.poison);
+                    bits = __shfl_sync(0xffffffffu, bits, 0);
+                    if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
+                    else w_in = __longlong_as_double((long long)bits);
+                }
+
+                // ---- the recursion, step by step (identical in every warp of the cluster) ---------------------------
+                // state: the resident u (total kappa), the node's weight w, and in lane j < kc the value of u at
+                // child j's token with its e_q (fp64, the same recursion as the vocabulary)
+                const bool live = !err && w_in > 0.0;
+                double w = live ? w_in : 0.0, kappa = Z_p;
+                bool dead = !live, is_q = false;      // is_q: a step with S = 0 at weight 1 showed that the state equals q
+                int nsteps = 0;
+                const int kce = min(kc, KMAX);
+                double ux = (lane < kce) ? W.cpm[lane] : 0.0;
+                const double eqx = (lane < kce) ? W.cqm[lane] : 0.0;
+                double *gs = TP.gseq + ((long long)b * P.N + a) * KMAX;
+                int acc = -1;
+                if (err && scribe) {
+                    // nothing below a faulty node is evaluated: every child gets weight / threshold 0
+                    for (int j = 0; j < kce; ++j) {
+                        const int c = W.child[j];
+                        if ((W.leaf_mask >> j) & 1u) { finish_leaf(c, 0.0); continue; }
+                        if (lane == 0) {
+                            NodeRec *rec = P.rec + (long long)b * P.N;
+                            if (trav) {
+                                rec[c].w_in = 0.0;
+                                *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
+                            } else {
+                                rec[c].thr = 0.0;
+                            }
                         }
                     }
-            }
-            for (int j = 0; j < kce && !err; ++j) {
-                // child j from the current state: P(x) = u(x) / kappa, q(x) = e_q(x) / Z_q
-                const double uxj = __shfl_sync(0xffffffffu, ux, j), eqj = __shfl_sync(0xffffffffu, eqx, j);
-                const double Pq = eqj * invZq;
-                const double Pp = is_q ? Pq : uxj / kappa;
-                double thr;
-                if (dead || !(Pp > 0.0)) thr = 0.0;
-                else if (!(Pq > 0.0)) thr = 1.0;
-                else thr = fmin(1.0, w * (Pp / Pq));
-                // Traversal: a weight within a rounding of 1 is 1.  The step after it is discontinuous at
-                // w = 1 when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
-                if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
-                if (scribe && lane == 0) {
-                    NodeRec *rec = P.rec + (long long)b * P.N;
-                    const int cj = W.child[j];
-                    if (trav) {
-                        // the child polls the published slot only; the record is read after all of the
-                        // sequence's arrivals (each fenced), so no fence is needed between the two stores
-                        rec[cj].w_in = thr;
-                        *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
-                            (unsigned long long)__double_as_longlong(thr);
+                }
+                for (int j = 0; j < kce && !err; ++j) {
+                    // child j from the current state: P(x) = u(x) / kappa, q(x) = e_q(x) / Z_q
+                    const double uxj = __shfl_sync(0xffffffffu, ux, j), eqj = __shfl_sync(0xffffffffu, eqx, j);
+                    const double Pq = eqj * invZq;
+                    const double Pp = is_q ? Pq : uxj / kappa;
+                    double thr;
+                    if (dead || !(Pp > 0.0)) thr = 0.0;
+                    else if (!(Pq > 0.0)) thr = 1.0;
+                    else thr = fmin(1.0, w * (Pp / Pq));
+                    // Traversal: a weight within a rounding of 1 is 1.  The step after it is discontinuous at
+                    // w = 1 when P = q (S = 0 gives weight 1 for w = 1 and weight 0 for any w < 1).
+                    if (trav && thr > 1.0 - WEIGHT_SNAP) thr = 1.0;
+                    if (scribe) {
+                        const int cj = W.child[j];
+                        if ((W.leaf_mask >> j) & 1u) {
+                            finish_leaf(cj, thr);
+                        } else if (lane == 0) {
+                            NodeRec *rec = P.rec + (long long)b * P.N;
+                            if (trav) {
+                                // the child polls the published slot only; the record is read after all of the
+                                // sequence's arrivals (each fenced), so no fence is needed between the two stores
+                                rec[cj].w_in = thr;
+                                *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
+                                    (unsigned long long)__double_as_longlong(thr);
+                            } else {
+                                rec[cj].thr = thr;
+                            }
+                        }
+                    }
+                    if (!trav && acc < 0 && (double)W.cu[j] < thr) {
+                        acc = W.child[j];
+                        if (!P.all_thr) {
+                            if (scribe)
+                                for (int jj = j + 1; jj < kce; ++jj) {
+                                    if ((W.leaf_mask >> jj) & 1u) finish_leaf(W.child[jj], CUDART_NAN);
+                                    else if (lane == 0) P.rec[(long long)b * P.N + W.child[jj]].thr = CUDART_NAN;
+                                }
+                            break;
+                        }
+                    }
+                    if (dead || is_q) continue;       // weight 0, or P = q (every further step has S = 0 again)
+                    // the step after rejecting child j: u <- (g u - e_q)+ , g = w Z_q / kappa
+                    const double g = __ddiv_rn(w * Z_q, kappa);
+                    const double v[1] = {warp_sum_once(step_sweep<NW>(es, nsm, tid, R, L, nl, g))};
+                    double tot[1], mine[1];
+                    cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                    if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
+                    ux = fmax(fma(g, ux, -eqx), 0.0);
+                    const double Sj = tot[0] * invZq;
+                    // A step whose mass is below 1e-13 of the weight before it counts as S = 0: P equals q, and what
+                    // is left is the rounding of g.
+                    if (Sj > RESIDUAL_FLOOR * w) {
+                        kappa = tot[0];
+                        if (trav) w = Sj / (Sj + (1.0 - w));
+                        if (scribe && lane == 0) gs[nsteps] = g;
+                        ++nsteps;
+                    } else if (w >= 1.0) {
+                        is_q = true;       // S = 0 with w = 1: the state is q itself (the stored u is no longer used)
+                        kappa = Z_q;
                     } else {
-                        rec[cj].thr = thr;
+                        dead = true;       // S = 0 with w < 1: the weight drops to 0 (Traversal only)
+                        w = 0.0;
                     }
                 }
-                if (!trav && acc < 0 && (double)W.cu[j] < thr) {
-                    acc = W.child[j];
-                    if (!P.all_thr) {
-                        if (scribe && lane == 0)
-                            for (int jj = j + 1; jj < kce; ++jj) P.rec[(long long)b * P.N + W.child[jj]].thr = CUDART_NAN;
-                        break;
+
+                // ---- the node's outcome -----------------------------------------------------------------------------
+                const double w_fin = (dead || err) ? 0.0 : w;
+                if (scribe) {
+                    if (lane == 0) {
+                        NodeRec &Rc = P.rec[(long long)b * P.N + a];
+                        Rc.O_p = (double)nr.O_p; Rc.Z_p = Z_p; Rc.O_q = (double)nr.O_q; Rc.Z_q = Z_q;
+                        Rc.kappa = (dead || err) ? 0.0 : kappa;
+                        Rc.nsteps = is_q ? STATE_IS_Q : nsteps;
+                        Rc.cut_p = nr.cut_p; Rc.cut_q = nr.cut_q;
+                        Rc.next_child = acc;
+                        Rc.status = err;
+                        Rc.bonus = -1; Rc.bonus_margin = 0.f;
+                        if (trav) { Rc.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) Rc.w_in = 1.0; }
+                        else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
                     }
+                    arrive_sequence(P, b);
                 }
-                if (dead || is_q) continue;       // weight 0, or P = q (every further step has S = 0 again)
-                // the step after rejecting child j: u <- (g u - e_q)+ , g = w Z_q / kappa
-                const double g = __ddiv_rn(w * Z_q, kappa);
-                const double v[1] = {warp_sum_once(step_sweep<NW>(es, nsm, tid, R, L, nl, g))};
+            } else {
+                // ---- FINISH: the accepted node back on chip, its recorded steps replayed, the bonus token drawn ---------
+                NodeRows nr;
+                nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+                nr.s_hi = (float)nr.s_d;
+                if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
+                nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
+                if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
+                const int nsteps = W.nsteps;
+                const bool is_q = nsteps == STATE_IS_Q;
+                nr.hq = nsteps != 0; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
+                set_list_thresholds(nr, W.Z_p, W.Z_q);
+                int nl;
+                float zs_p, zs_q;
+                pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
+                double part = (double)zs_p + (lane < nl ? L.ep[lane] : 0.0);
+                if (is_q) part = (double)zs_q + (lane < nl ? L.eq[lane] : 0.0);
+                for (int j = 0; j < nsteps; ++j) part = step_sweep<NW>(es, nsm, tid, R, L, nl, W.cpm[j]);
+                const double v[1] = {warp_sum_once(part)};
                 double tot[1], mine[1];
                 cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
-                ux = fmax(fma(g, ux, -eqx), 0.0);
-                const double Sj = tot[0] * invZq;
-                // A step whose mass is below 1e-13 of the weight before it counts as S = 0: P equals q, and what
-                // is left is the rounding of g.
-                if (Sj > RESIDUAL_FLOOR * w) {
-                    kappa = tot[0];
-                    tot_r = mine[0];
-                    if (trav) w = Sj / (Sj + (1.0 - w));
-                    if (gs && scribe && lane == 0) gs[nsteps] = g;
-                    ++nsteps;
-                } else if (w >= 1.0) {
-                    is_q = true;       // S = 0 with w = 1: the state is q itself (the stored u is no longer used)
-                    tot_r = Zr_q;
-                    kappa = Z_q;
-                } else {
-                    dead = true;       // S = 0 with w < 1: the weight drops to 0 (Traversal only)
-                    w = 0.0;
+                int ferr = (poisoned || *(volatile int *)&S.poison) ? SPEC_DEV_TIMEOUT : 0;
+                double tau = 0.0;
+                int owner = -1;
+                if (!ferr) {
+                    const double target = (double)W.ub_a * tot[0];
+                    owner = pick_lane(lane < C ? mine[0] : 0.0, target, tau);
+                    if (owner < 0) ferr = SPEC_DEV_NONFINITE;
                 }
-            }
-
-            // ---- the node's outcome -----------------------------------------------------------------------------
-            const double w_fin = (dead || err) ? 0.0 : w;
-            bool want_bonus;
-            if (trav) want_bonus = (a == 0) || ((double)W.u_a < w_fin);
-            else want_bonus = acc < 0;
-            if (dead || err) want_bonus = false;
-            int owner = -1;
-            double tau = 0.0, E_tot = 0.0;
-            if (want_bonus && !hq) {
-                // a childless node: the totals of u_0 = e_p per rank (pass 1 summed them already)
-                const double v[1] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0))};
-                double tot[1], mine[1];
-                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
-                tot_r = mine[0];
-                kappa = tot[0];
-                if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; want_bonus = false; }
-            }
-            if (want_bonus) {
-                E_tot = warp_sum_once(lane < C ? tot_r : 0.0);
-                const double target = (double)W.ub_a * E_tot;
-                owner = pick_lane(lane < C ? tot_r : 0.0, target, tau);
-            }
-            if (scribe) {
-                if (lane == 0) {
-                    NodeRec &Rc = P.rec[(long long)b * P.N + a];
-                    Rc.O_p = (double)nr.O_p; Rc.Z_p = Z_p; Rc.O_q = (double)nr.O_q; Rc.Z_q = Z_q;
-                    Rc.kappa = (dead || err) ? 0.0 : kappa;
-                    Rc.nsteps = is_q ? STATE_IS_Q : nsteps;
-                    Rc.cut_p = nr.cut_p; Rc.cut_q = nr.cut_q;
-                    Rc.next_child = acc;
-                    Rc.status = err;
-                    if (trav) { Rc.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) Rc.w_in = 1.0; }
-                    else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
-                    if (owner < 0) { Rc.bonus = -1; Rc.bonus_margin = 0.f; }
+                int role = 0, tokn = -1;
+                float mg = 0.f;
+                if (ferr) {
+                    role = (scribe && lane == 0) ? (ferr == SPEC_DEV_TIMEOUT ? 3 : 2) : 0;
+                } else if (owner == (int)rank) {
+                    const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl, is_q, tau);
+                    role = bf.role;
+                    tokn = (int)(tok0 + bf.token);
+                    mg = (float)(bf.edge / tot[0]);
                 }
-                arrive_sequence(P, b, owner < 0 ? 2u : 1u);
-            }
-
-            // ---- bonus token: inverse CDF over the owner CTA's share of the state ----------------------------------
-            if (owner == (int)rank) {
-                const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl, is_q, tau);
-                if (bf.role) {
-                    NodeRec &Rc = P.rec[(long long)b * P.N + a];
-                    Rc.bonus = bf.role == 1 ? (int)(tok0 + bf.token) : (bf.role == 3 ? BONUS_TIMEOUT : -1);
-                    Rc.bonus_margin = bf.role == 1 ? (float)(bf.edge / E_tot) : 0.f;
+                if (role == 1) {
+                    const int len = __ldcg(P.out.accept_len + b);
+                    P.out.bonus_token[b] = tokn;
+                    P.out.out_tokens[(long long)b * P.N + len] = tokn;
+                    if (P.out.margin) P.out.margin[(long long)b * (P.N + 1) + P.N] = mg;
+                } else if (role >= 2) {
+                    P.out.status[b] = role == 3 ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE;
+                    P.out.accepted_node[b] = -1; P.out.accept_len[b] = -1; P.out.bonus_token[b] = -1;
+                    int *ot = P.out.out_tokens + (long long)b * P.N;
+                    for (int i = 0; i < P.N; ++i) ot[i] = -1;
                 }
-                // the arrival is made by lane 0 of the warp that holds the reporting thread
-                __syncwarp();
-                if (__any_sync(0xffffffffu, bf.role != 0)) arrive_sequence(P, b, 1u);
             }
             // the scalars block may be rewritten
             __syncwarp();

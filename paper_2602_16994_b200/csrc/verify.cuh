@@ -52,7 +52,8 @@ constexpr int NSMAX = 16;    // ring stages
 constexpr int NWMAX = 15;    // consumer warps
 constexpr int OMIN = -(1 << 30);
 constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
-constexpr int BONUS_TIMEOUT = -2;   // NodeRec::bonus of a node whose bonus search gave up on a wait
+constexpr int FIN_PENDING = -1;     // VParams::fin of a sequence whose nodes are not all done
+constexpr int FIN_FAULTY = -2;      // ... of a sequence with a device-detected fault: no bonus draw
 // A residual step whose mass is below this fraction of the mass before it is treated as S = 0: where P
 // equals q (the same row twice, two one-token nuclei on the same token) the exact difference is 0 and
 // the computed one a few 1e-16 of the mass (the rounding of the coefficient g).
@@ -83,7 +84,8 @@ struct VParams {
     const float *u_accept, *u_bonus;
     NodeRec *rec;
     unsigned long long *w_pub;   // [B*N] weight handed to a node by its parent (Traversal), W_PENDING until known
-    unsigned int *done;          // [B] arrivals per sequence (two per node); the last one writes the outputs
+    unsigned int *done;          // [B] arrivals per sequence (one per node); the last one selects the accepted node
+    int *fin;                    // [B] the accepted node once it is selected (FIN_PENDING before, FIN_FAULTY for a faulty sequence)
     SpecOut out;
 };
 
@@ -645,8 +647,10 @@ __device__ __forceinline__ BonusFind bonus_search(double (*wtile)[TMAX], uint64_
 }
 
 // ------------------------------------------------------------------------------------------------
-// writing the outputs of one sequence: run by the whole warp whose lane made the last arrival
+// selecting the accepted node of one sequence: run by the whole warp whose lane made the last arrival
 // ------------------------------------------------------------------------------------------------
+// Writes every output of the sequence except the bonus token (accepted node, length, path tokens, status,
+// the per-node diagnostics) and publishes the accepted node in P.fin for the sequence's FINISH item.
 __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
 {
     const int lane = threadIdx.x & 31;
@@ -730,19 +734,16 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
         }
         if (acc < 0) status = SPEC_DEV_TOPOLOGY;
     }
-    int bonus = acc >= 0 ? __ldcg(&rec[acc].bonus) : -1;
-    if (acc >= 0 && bonus < 0 && !status) status = bonus == BONUS_TIMEOUT ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE;
-    if (status) { acc = -1; len = -1; bonus = -1; }
+    if (status) { acc = -1; len = -1; }
     int *ot = P.out.out_tokens + (long long)b * N;
     for (int i = lane; i < N; i += 32) ot[i] = -1;
     __syncwarp();
     if (lane == 0) {
         P.out.accepted_node[b] = acc;
         P.out.accept_len[b] = len;
-        P.out.bonus_token[b] = bonus;
+        P.out.bonus_token[b] = -1;         // the FINISH item draws it
         P.out.status[b] = status;
         if (acc >= 0) {
-            ot[len] = bonus;
             int i = len;
             for (int x = acc; x != 0 && i > 0; x = parent[x]) ot[--i] = token[x];
         }
@@ -755,21 +756,27 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
         float *mg = P.out.margin + (long long)b * (N + 1);
         for (int i = lane; i < N; i += 32)
             mg[i] = i == 0 ? CUDART_NAN_F : (float)fabs((double)ua[i] - __ldcg(&rec[i].thr));
-        if (lane == 0) mg[N] = acc >= 0 ? __ldcg(&rec[acc].bonus_margin) : CUDART_NAN_F;
+        if (lane == 0) mg[N] = CUDART_NAN_F;
+    }
+    // publication: everything above is visible to whoever sees the accepted node
+    __syncwarp();
+    if (lane == 0) {
+        __threadfence();
+        *(volatile int *)(P.fin + b) = status ? FIN_FAULTY : acc;
     }
 }
 
-// `count` arrivals of a node at its sequence, made by lane 0 of a converged warp; the warp that makes
-// the last of the 2N arrivals writes the sequence's outputs.
-__device__ __forceinline__ void arrive_sequence(const VParams &P, int b, unsigned count)
+// One arrival of a node at its sequence, made by lane 0 of a converged warp; the warp that makes the
+// last of the N arrivals selects the accepted node.
+__device__ __forceinline__ void arrive_sequence(const VParams &P, int b)
 {
     int last = 0;
     if ((threadIdx.x & 31) == 0) {
         // release: the node's record (written by this warp, ordered before by __syncwarp where another
         // lane wrote it) is visible to whoever sees the count; acquire: the last arrival sees all records
         unsigned prev;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(P.done + b), "r"(count) : "memory");
-        last = (prev + count == 2u * (unsigned)P.N) ? 1 : 0;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(P.done + b), "r"(1u) : "memory");
+        last = (prev + 1u == (unsigned)P.N) ? 1 : 0;
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) finalize_sequence(P, b);
