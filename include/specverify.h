@@ -170,6 +170,47 @@ int32_t spec_verify_traversal(const SpecIn *in, const SpecOut *out, void *ws, in
                               void *stream);
 
 /*
+ * Offline analysis of a batch of draft trees (Section 5 and Appendices C, D): for every node with
+ * children, from its sampling distributions p, q (same transform as the verifiers) and its child list,
+ *   acceptance  [B,N,4] acceptance rates alpha(f) of Definition 5.1 with k = the node's number of
+ *               children: NSS (Algorithm 6), Naive (Algorithm 7), SpecTr (Algorithm 8), SpecInfer
+ *               (Algorithm 9);
+ *   divergence  [B,N,3] L1 distance sum |p - q| (Section 5), KL(p||q), KL(q||p) in nats (the selector's
+ *               scalar features, Section 6; +inf where the second law has no mass under the first);
+ *   branch      [5][B,N] branching probability B(f, ch(parent), token) of Definition 5.3 of moving from
+ *               the parent into the node, for f = NSS (Algorithm 11), Naive (12), SpecTr (13), SpecInfer
+ *               with children tried in list order (what spec_verify_specinfer runs), SpecInfer with the
+ *               next child picked uniformly (Algorithm 14; NaN for more than 10 children); root: 1; a
+ *               child whose token an earlier sibling carries is never moved to: 0;
+ *   reach       [5][B,N] product of the branching probabilities along the node's path;
+ *   block_eff   [5][B]  sum of reach over the tree's nodes = E[tau + 1 | tree], the inner sum of
+ *               equation (3) (average it over sampled trees for the paper's estimator).
+ * Rows of childless nodes are NaN in acceptance / divergence.  All outputs are device pointers, all
+ * required.  `ws`: spec_analysis_workspace_bytes() bytes.  u_accept / u_bonus of `in` must be valid
+ * but do not influence the outputs.  SpecTr's rho* is found by 40 bisection steps on [1, k].
+ */
+typedef struct {
+    float *acceptance;
+    float *divergence;
+    float *branch;
+    float *reach;
+    float *block_eff;
+} SpecAnalysisOut;
+int32_t spec_analysis_workspace_bytes(const SpecIn *in, int64_t *bytes);
+int32_t spec_tree_analysis(const SpecIn *in, const SpecAnalysisOut *out, void *ws, int64_t ws_bytes, void *stream);
+
+/*
+ * Forward-pass time of delayed-expansion actions (Appendix E, equation (8)): for action a = (K, L1, L2)
+ * at context length ctx,
+ *   T_hat[a] = sum_{j<L1} t_q(ctx + j) + sum_{j<L2} t_q(ctx + L1 + j K) + t_p(ctx + L1 + K L2),
+ * t_q / t_p: measured draft / target forward times per context length (tables of n_len doubles; a length
+ * beyond the table uses its last entry).  actions [n_actions,3] int32, T_hat [n_actions] double; all
+ * device pointers.
+ */
+int32_t spec_latency_model(const double *t_q, const double *t_p, int32_t n_len, int32_t ctx, const int32_t *actions,
+                           int32_t n_actions, double *T_hat, void *stream);
+
+/*
  * Inverse-CDF draw (the "Sample Y ~ p" steps of Algorithms 1-4) from R rows of non-negative
  * weights that need not be normalised: token[r] = smallest t with w_0 + ... + w_t > u[r] * sum(w).
  *   weights [R,V] float contiguous, u [R] in [0,1), token [R] (-1 for an all-zero row),

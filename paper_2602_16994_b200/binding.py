@@ -26,7 +26,8 @@ ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR
           -4: "SPEC_ERR_PARAM", -5: "SPEC_ERR_WORKSPACE", -6: "SPEC_ERR_UNSUPPORTED", -7: "SPEC_ERR_CUDA"}
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
            "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
-           "spec_verify_specinfer_static", "spec_kernel_launches")
+           "spec_verify_specinfer_static", "spec_kernel_launches", "spec_analysis_workspace_bytes",
+           "spec_tree_analysis", "spec_latency_model")
 
 
 class SpecIn(C.Structure):
@@ -48,6 +49,13 @@ class SpecOut(C.Structure):
         ("margin", C.c_void_p),
     ]
 
+
+class SpecAnalysisOut(C.Structure):
+    _fields_ = [("acceptance", C.c_void_p), ("divergence", C.c_void_p), ("branch", C.c_void_p),
+                ("reach", C.c_void_p), ("block_eff", C.c_void_p)]
+
+
+SOLVERS = ("nss", "naive", "spectr", "specinfer", "specinfer_uniform")     # order of the `branch` outputs
 
 _lib = None
 
@@ -84,6 +92,13 @@ def load_library(path: str = LIB_PATH):
     lib.spec_verify_host.restype = C.c_int32
     lib.spec_verify_host.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_int32, C.c_void_p, C.c_int64,
                                      C.c_void_p]
+    lib.spec_analysis_workspace_bytes.restype = C.c_int32
+    lib.spec_analysis_workspace_bytes.argtypes = [C.POINTER(SpecIn), C.POINTER(C.c_int64)]
+    lib.spec_tree_analysis.restype = C.c_int32
+    lib.spec_tree_analysis.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecAnalysisOut), C.c_void_p, C.c_int64, C.c_void_p]
+    lib.spec_latency_model.restype = C.c_int32
+    lib.spec_latency_model.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
+                                       C.c_void_p]
     _lib = lib
     return lib
 
@@ -303,6 +318,51 @@ class PreparedVerify:
         if rc != 0:
             _check(rc, "spec_verify_" + self.name)
         return self.outputs
+
+
+@dataclass
+class AnalysisOutputs:
+    acceptance: torch.Tensor     # [B,N,4]: NSS, Naive, SpecTr, SpecInfer
+    divergence: torch.Tensor     # [B,N,3]: L1, KL(p||q), KL(q||p)
+    branch: torch.Tensor         # [5,B,N], order of SOLVERS
+    reach: torch.Tensor          # [5,B,N]
+    block_eff: torch.Tensor      # [5,B]
+
+
+def tree_analysis(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0, top_k=0,
+                  top_p=1.0, temperature_per_seq=None, stream=None) -> AnalysisOutputs:
+    """Acceptance rates, divergences, branching probabilities and block efficiency of a batch of trees."""
+    lib = load_library()
+    si, keep = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+                        temperature_per_seq)
+    B, N = si.B, si.N
+    dev = target_logits.device
+    f32 = dict(dtype=torch.float32, device=dev)
+    out = AnalysisOutputs(torch.empty((B, N, 4), **f32), torch.empty((B, N, 3), **f32), torch.empty((5, B, N), **f32),
+                          torch.empty((5, B, N), **f32), torch.empty((5, B), **f32))
+    n = C.c_int64()
+    _check(lib.spec_analysis_workspace_bytes(C.byref(si), C.byref(n)), "spec_analysis_workspace_bytes")
+    ptr, size = _ws_for(dev).get(int(n.value))
+    so = SpecAnalysisOut(_ptr(out.acceptance), _ptr(out.divergence), _ptr(out.branch), _ptr(out.reach),
+                         _ptr(out.block_eff))
+    _check(lib.spec_tree_analysis(C.byref(si), C.byref(so), ptr, size, _stream_ptr(stream)), "spec_tree_analysis")
+    return out
+
+
+def latency_model(t_q, t_p, ctx, actions, stream=None):
+    """Equation (8): forward-pass time of every action (K, L1, L2) at context length ``ctx`` (device tensors:
+    t_q / t_p float64 [n_len], actions int32 [A,3]); returns float64 [A]."""
+    lib = load_library()
+    for name, t, dt in (("t_q", t_q, torch.float64), ("t_p", t_p, torch.float64), ("actions", actions, torch.int32)):
+        _require_cuda(t, name)
+        if t.dtype != dt or not t.is_contiguous():
+            raise RuntimeError(f"{name} must be a contiguous {dt} tensor")
+    if t_q.numel() != t_p.numel() or actions.dim() != 2 or actions.shape[1] != 3:
+        raise RuntimeError("t_q and t_p must have the same length, actions must be [A,3]")
+    out = torch.empty(actions.shape[0], dtype=torch.float64, device=t_q.device)
+    _check(lib.spec_latency_model(_ptr(t_q), _ptr(t_p), t_q.numel(), int(ctx), _ptr(actions), actions.shape[0],
+                                  _ptr(out), _stream_ptr(stream)), "spec_latency_model")
+    return out
 
 
 def tree_probs(logits, which=0, temperature=1.0, top_k=0, top_p=1.0, temperature_per_seq=None,

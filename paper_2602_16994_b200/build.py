@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 SRC = [os.path.join(HERE, "csrc", "specverify.cu")]
-DEPS = [os.path.join(HERE, "csrc", f) for f in ("common.cuh", "verify.cuh", "rowops.cuh", "cut.cuh", "rowstat.cuh", "stream.cuh", "walk.cuh", "tree.cuh", "trunc.cuh")]
+DEPS = [os.path.join(HERE, "csrc", f) for f in ("common.cuh", "verify.cuh", "rowops.cuh", "cut.cuh", "rowstat.cuh", "stream.cuh", "walk.cuh", "tree.cuh", "trunc.cuh", "analysis.cuh")]
 LIB = os.path.join(HERE, "libspecverify.so")
 HEADERS = [os.path.join(ROOT, "include", "specverify.h")]
 

@@ -12,6 +12,7 @@
 #include <atomic>
 #include <mutex>
 
+#include "analysis.cuh"
 #include "common.cuh"
 #include "cut.cuh"
 #include "rowops.cuh"
@@ -295,10 +296,10 @@ int resident_clusters(K kernel, int C, int threads, int smem)
     return n;
 }
 
-template <int DT, int NW>
+template <int DT, int NW, bool AN>
 int launch_tree(const VPlan &pl, TParams &tp, cudaStream_t st)
 {
-    auto kernel = spec_tree_kernel<DT, NW>;
+    auto kernel = spec_tree_kernel<DT, NW, AN>;
     int rc = prepare_kernel(kernel, pl.C, pl.smem);
     if (rc) return rc;
     const int threads = (NW + 1) * 32;
@@ -467,6 +468,40 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
     return bf ? launch_walk<SPEC_BF16, 15, 1>(pl, wp, st) : launch_walk<SPEC_F32, 15, 1>(pl, wp, st);
 }
 
+void fill_tparams(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl, int mode,
+                  TParams &tp)
+{
+    VParams &vp = tp.v;
+    vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
+    vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
+    vp.slice_len = pl.slice_len; vp.NS = pl.NS; vp.nsm = pl.nsm;
+    vp.off_x = pl.off_x; vp.off_list = pl.off_list; vp.off_es = pl.off_es; vp.off_ring = pl.off_ring;
+    vp.zp = in->target_logits; vp.zq = in->draft_logits;
+    vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
+    vp.parent = in->parent; vp.token = in->token;
+    vp.T = in->temperature; vp.T_seq = in->temperature_per_seq;
+    vp.u_accept = in->u_accept; vp.u_bonus = in->u_bonus;
+    vp.rec = (NodeRec *)(w + L.rec);
+    vp.w_pub = (unsigned long long *)(w + L.pub);
+    vp.done = (unsigned int *)(w + L.done);
+    vp.fin = (int *)(w + L.fin);
+    vp.out = *out;
+    tp.part = (const RowPart *)(w + L.stat);
+    tp.gseq = (double *)(w + L.gseq);
+    tp.ticket = (unsigned int *)(w + L.ticket);
+}
+
+int launch_tree_any(const SpecIn *in, const VPlan &pl, TParams &tp, bool analysis, cudaStream_t st)
+{
+    const bool bf = in->logits_dtype == SPEC_BF16;
+    if (analysis) {
+        if (pl.NW == 7) return bf ? launch_tree<SPEC_BF16, 7, true>(pl, tp, st) : launch_tree<SPEC_F32, 7, true>(pl, tp, st);
+        return bf ? launch_tree<SPEC_BF16, 15, true>(pl, tp, st) : launch_tree<SPEC_F32, 15, true>(pl, tp, st);
+    }
+    if (pl.NW == 7) return bf ? launch_tree<SPEC_BF16, 7, false>(pl, tp, st) : launch_tree<SPEC_F32, 7, false>(pl, tp, st);
+    return bf ? launch_tree<SPEC_BF16, 15, false>(pl, tp, st) : launch_tree<SPEC_F32, 15, false>(pl, tp, st);
+}
+
 int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream, int mode,
                   bool parts = true)
 {
@@ -498,27 +533,9 @@ int verify_common(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_byt
     rc = row_statistics(in, out, w, L, trunc, parts, st, true);
     if (rc) return rc;
     TParams tp = {};
+    fill_tparams(in, out, w, L, pl, mode, tp);
     VParams &vp = tp.v;
-    vp.B = in->B; vp.N = in->N; vp.V = in->V; vp.C = pl.C; vp.mode = mode;
-    vp.all_thr = (out->node_thr != nullptr || out->margin != nullptr) ? 1 : 0;
-    vp.slice_len = pl.slice_len; vp.NS = pl.NS; vp.nsm = pl.nsm;
-    vp.off_x = pl.off_x; vp.off_list = pl.off_list; vp.off_es = pl.off_es; vp.off_ring = pl.off_ring;
-    vp.zp = in->target_logits; vp.zq = in->draft_logits;
-    vp.seq_stride = in->seq_stride; vp.node_stride = in->node_stride; vp.topo_stride = in->topo_seq_stride;
-    vp.parent = in->parent; vp.token = in->token;
-    vp.T = in->temperature; vp.T_seq = in->temperature_per_seq;
-    vp.u_accept = in->u_accept; vp.u_bonus = in->u_bonus;
-    vp.rec = (NodeRec *)(w + L.rec);
-    vp.w_pub = (unsigned long long *)(w + L.pub);
-    vp.done = (unsigned int *)(w + L.done);
-    vp.fin = (int *)(w + L.fin);
-    vp.out = *out;
-    tp.part = (const RowPart *)(w + L.stat);
-    tp.gseq = (double *)(w + L.gseq);
-    tp.ticket = (unsigned int *)(w + L.ticket);
-    const bool bf = in->logits_dtype == SPEC_BF16;
-    if (pl.NW == 7) rc = bf ? launch_tree<SPEC_BF16, 7>(pl, tp, st) : launch_tree<SPEC_F32, 7>(pl, tp, st);
-    else rc = bf ? launch_tree<SPEC_BF16, 15>(pl, tp, st) : launch_tree<SPEC_F32, 15>(pl, tp, st);
+    rc = launch_tree_any(in, pl, tp, false, st);
     if (rc) return rc;
     if (out->residual) {
         RParams rp = {};
@@ -644,6 +661,89 @@ int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void 
     rc = static_ws_address(&ws);
     if (rc) return rc;
     return verify_common(in, out, ws, STATIC_WS_BYTES, stream, MODE_SPECINFER, false);
+}
+
+// analysis workspace: the verifiers' layout | per-node scalars | scratch for the decision outputs nobody reads
+struct AnLayout {
+    int64_t an, acc, len, toks, bonus, status, total;
+};
+static AnLayout an_layout(const SpecIn *in)
+{
+    AnLayout A;
+    const int64_t nodes = (int64_t)in->B * in->N;
+    int64_t o = up256(ws_layout(in).total);
+    A.an = o; o += up256(nodes * (int64_t)sizeof(AnRec));
+    A.acc = o; o += up256((int64_t)in->B * 4);
+    A.len = o; o += up256((int64_t)in->B * 4);
+    A.toks = o; o += up256(nodes * 4);
+    A.bonus = o; o += up256((int64_t)in->B * 4);
+    A.status = o; o += up256((int64_t)in->B * 4);
+    A.total = o;
+    return A;
+}
+
+int32_t spec_analysis_workspace_bytes(const SpecIn *in, int64_t *bytes)
+{
+    if (!in || !bytes) return SPEC_ERR_NULL;
+    if (in->B <= 0 || in->N <= 0 || in->N > SPEC_MAX_NODES || (long long)in->B * in->N > (1ll << 24))
+        return SPEC_ERR_SHAPE;
+    *bytes = an_layout(in).total;
+    return SPEC_OK;
+}
+
+int32_t spec_tree_analysis(const SpecIn *in, const SpecAnalysisOut *out, void *ws, int64_t ws_bytes, void *stream)
+{
+    int rc = check_in(in, true);
+    if (rc) return rc;
+    if (!out || !out->acceptance || !out->divergence || !out->branch || !out->reach || !out->block_eff) return SPEC_ERR_NULL;
+    const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
+    const WsLayout L = ws_layout(in);
+    const AnLayout A = an_layout(in);
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < A.total) return SPEC_ERR_WORKSPACE;
+    VPlan pl;
+    if (!make_vplan(in->V, in->logits_dtype, &pl)) return SPEC_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *w = (unsigned char *)ws;
+    const int64_t nodes = (int64_t)in->B * in->N;
+    // outputs start as NaN (all-ones), the per-node scalars as "no children"
+    bool ok = true;
+    ok &= cudaMemsetAsync(out->acceptance, 0xFF, (size_t)nodes * 16, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(out->divergence, 0xFF, (size_t)nodes * 12, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(out->branch, 0xFF, (size_t)nodes * 4 * analysis::NSOLVER, st) == cudaSuccess;
+    ok &= cudaMemsetAsync(w + A.an, 0, (size_t)nodes * sizeof(AnRec), st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SPEC_ERR_CUDA; }
+    SpecOut so = {};
+    so.accepted_node = (int32_t *)(w + A.acc); so.accept_len = (int32_t *)(w + A.len);
+    so.out_tokens = (int32_t *)(w + A.toks); so.bonus_token = (int32_t *)(w + A.bonus);
+    so.status = (int32_t *)(w + A.status);
+    rc = row_statistics(in, &so, w, L, trunc, true, st, true);
+    if (rc) return rc;
+    TParams tp = {};
+    fill_tparams(in, &so, w, L, pl, MODE_SPECINFER, tp);
+    tp.v.all_thr = 1;
+    tp.an = (AnRec *)(w + A.an); tp.an_acc = out->acceptance; tp.an_div = out->divergence;
+    rc = launch_tree_any(in, pl, tp, true, st);
+    if (rc) return rc;
+    analysis::BParams bp = {in->B, in->N, in->parent, in->token, in->topo_seq_stride, tp.an, out->acceptance, out->branch};
+    analysis::spec_branch_kernel<<<(unsigned)((nodes + 3) / 4), 128, 0, st>>>(bp);
+    g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
+    analysis::RParams rp = {in->B, in->N, in->parent, in->topo_seq_stride, out->branch, out->reach, out->block_eff};
+    analysis::spec_reach_kernel<<<(unsigned)((analysis::NSOLVER * in->B + 127) / 128), 128, 0, st>>>(rp);
+    g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    return SPEC_OK;
+}
+
+int32_t spec_latency_model(const double *t_q, const double *t_p, int32_t n_len, int32_t ctx, const int32_t *actions,
+                           int32_t n_actions, double *T_hat, void *stream)
+{
+    if (!t_q || !t_p || !actions || !T_hat) return SPEC_ERR_NULL;
+    if (n_len <= 0 || n_actions <= 0 || ctx < 0) return SPEC_ERR_SHAPE;
+    analysis::LParams lp = {t_q, t_p, n_len, ctx, n_actions, actions, T_hat};
+    analysis::spec_latency_kernel<<<(unsigned)((n_actions + 127) / 128), 128, 0, (cudaStream_t)stream>>>(lp);
+    g_kernel_launches.fetch_add(1, std::memory_order_relaxed);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    return SPEC_OK;
 }
 
 int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *row_stats, void *ws,

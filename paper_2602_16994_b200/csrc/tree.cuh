@@ -31,6 +31,7 @@
 // the sequence's FINISH item brings that one node back on chip, replays its recorded steps (no
 // exchange: the coefficients are known) and draws the bonus token by the inverse-CDF search.
 #pragma once
+#include "analysis.cuh"
 #include "stream.cuh"
 #include "verify.cuh"
 
@@ -41,6 +42,10 @@ struct TParams {
     const RowPart *part;      // [B*N*2] statistics of every row the verifier reads
     double *gseq;             // [B*N][KMAX]: the step coefficients g_j of every node
     unsigned int *ticket;     // item counter (0 at launch)
+    // analysis instantiation only (SpecInfer mode, every threshold evaluated)
+    AnRec *an;                // [B*N] per-node scalars for the branching probabilities
+    float *an_acc;            // [B,N,4] acceptance rates: NSS, Naive, SpecTr written here (SpecInfer by spec_branch_kernel)
+    float *an_div;            // [B,N,3] L1, KL(p||q), KL(q||p)
 };
 
 // ITEM_LEAF: a childless root (a tree of one node); other childless nodes are never items
@@ -100,7 +105,10 @@ __device__ __forceinline__ unsigned long long poll_weight(const unsigned long lo
     return bits;
 }
 
-template <int DT, int NW>
+// AN: the analysis instantiation (read-only sweeps for acceptance rates and divergences, SpecTr's bisection,
+// the per-node scalars of the branching probabilities) -- a separate instantiation, so that the verifiers'
+// kernels carry none of it
+template <int DT, int NW, bool AN>
 __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kernel(const TParams TP)
 {
     const VParams &P = TP.v;
@@ -494,7 +502,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 // ---- pass 1: e = 2^(z s - O) of both rows, resident; dominant tokens to the exact lists -------------
                 int nl;
                 float zs_p, zs_q;
-                pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
+                KlSums kls = {0.f, 0.f, 0.f, 0.f};
+                pass1<DT, NW, AN>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q, &kls);
                 if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
 
                 // ---- the rows' normalisers from what is resident (one exchange) -----------------------------------
@@ -518,6 +527,65 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     bits = __shfl_sync(0xffffffffu, bits, 0);
                     if (bits == W_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; w_in = 0.0; }
                     else w_in = __longlong_as_double((long long)bits);
+                }
+
+                // ---- offline analysis on the untouched rows (read-only sweeps, totals identical in every warp) ----------
+                double an_rho = 1.0, an_beta = 0.0, an_pacc = 0.0, an_sres = 0.0;
+                if (AN && !err) {
+                    const double ip = __drcp_rn(Z_p), iq = invZq;
+                    const double kd = (double)kc;
+                    auto sweep2 = [&](auto f, double &t0, double &t1) {
+                        double o0, o1;
+                        reduce_sweep<NW>(es, nsm, tid, R, L, nl, f, o0, o1);
+                        const double v[2] = {warp_sum_once(o0), warp_sum_once(o1)};
+                        double tot[2], mine[2];
+                        cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                        t0 = tot[0]; t1 = tot[1];
+                    };
+                    double l1, smin, klpq, klqp, nss, naive2;
+                    sweep2(FnL1Min{(float)ip, (float)iq, ip, iq}, l1, smin);
+                    {
+                        // KL(p||q) = ln 2 (sum e_p x_p - sum e_p x_q) / Z_p - ln Z_p + ln Z_q, and the mirror image
+                        const double v1[2] = {warp_sum_once((double)kls.pp), warp_sum_once((double)kls.pq)};
+                        const double v2[2] = {warp_sum_once((double)kls.qq), warp_sum_once((double)kls.qp)};
+                        double t1[2], t2[2], mine[2];
+                        cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v1, t1, mine);
+                        cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v2, t2, mine);
+                        const double lz = log(Z_p) - log(Z_q);
+                        klpq = 0.6931471805599453 * (t1[0] - t1[1]) * ip - lz;
+                        klqp = 0.6931471805599453 * (t2[0] - t2[1]) * iq + lz;
+                    }
+                    sweep2(FnNssNaive{(float)ip, (float)iq, ip, iq, (float)kd, kd}, nss, naive2);
+                    // SpecTr's division factor: root of 1 - (1 - beta)^k - rho beta on [1, k] by bisection (Appendix B)
+                    double lo = 1.0, hi = kd, dummy;
+                    if (kc > 1) {
+                        for (int it = 0; it < 40; ++it) {
+                            const double mid = 0.5 * (lo + hi), ipr = ip / mid;
+                            double beta;
+                            sweep2(FnBeta{(float)ipr, (float)iq, ipr, iq}, beta, dummy);
+                            const double f = (1.0 - pow(1.0 - beta, kd)) - mid * beta;
+                            if (f > 0.0) lo = mid; else hi = mid;
+                        }
+                        an_rho = 0.5 * (lo + hi);
+                    }
+                    {
+                        const double ipr = ip / an_rho;
+                        sweep2(FnBeta{(float)ipr, (float)iq, ipr, iq}, an_beta, dummy);
+                    }
+                    an_pacc = 1.0 - pow(1.0 - an_beta, kd);
+                    const double gamma = an_beta > 0.0 ? an_pacc / an_beta : 0.0;
+                    const double ib = an_beta < 1.0 ? 1.0 / (1.0 - an_beta) : 0.0;
+                    double sacc;
+                    sweep2(FnSpecTrRes{(float)ip, (float)iq, (float)(1.0 / an_rho), (float)gamma, (float)ib, (float)kd,
+                                       ip, iq, 1.0 / an_rho, gamma, ib, kd}, an_sres, sacc);
+                    if (*(volatile int *)&S.poison) err = SPEC_DEV_TIMEOUT;
+                    if (scribe && lane == 0 && !err) {
+                        float *ao = TP.an_acc + ((long long)b * P.N + a) * 4, *dv = TP.an_div + ((long long)b * P.N + a) * 3;
+                        ao[0] = (float)nss;
+                        ao[1] = (float)(smin + naive2);
+                        ao[2] = (float)(an_pacc + (1.0 - an_pacc) * (an_sres > 0.0 ? sacc / an_sres : 0.0));
+                        dv[0] = (float)l1; dv[1] = (float)klpq; dv[2] = (float)klqp;
+                    }
                 }
 
                 // ---- the recursion, step by step (identical in every warp of the cluster) ---------------------------
@@ -553,6 +621,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     const double uxj = __shfl_sync(0xffffffffu, ux, j), eqj = __shfl_sync(0xffffffffu, eqx, j);
                     const double Pq = eqj * invZq;
                     const double Pp = is_q ? Pq : uxj / kappa;
+                    if (AN && scribe && lane < kce) {
+                        // round j's acceptance probability of every child's token: min(1, p_j(x_t) / q(x_t))
+                        const double q_t = eqx * invZq, p_t = is_q ? q_t : ux / kappa;
+                        TP.an[(long long)b * P.N + a].A[j][lane] =
+                            !(p_t > 0.0) ? 0.0 : (!(q_t > 0.0) ? 1.0 : fmin(1.0, p_t / q_t));
+                    }
                     double thr;
                     if (dead || !(Pp > 0.0)) thr = 0.0;
                     else if (!(Pq > 0.0)) thr = 1.0;
@@ -588,6 +662,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                             break;
                         }
                     }
+                    if (AN && scribe && lane == 0 && (dead || is_q)) TP.an[(long long)b * P.N + a].S[j] = 0.0;
                     if (dead || is_q) continue;       // weight 0, or P = q (every further step has S = 0 again)
                     // the step after rejecting child j: u <- (g u - e_q)+ , g = w Z_q / kappa
                     const double g = __ddiv_rn(w * Z_q, kappa);
@@ -597,6 +672,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     if (*(volatile int *)&S.poison) { err = SPEC_DEV_TIMEOUT; break; }
                     ux = fmax(fma(g, ux, -eqx), 0.0);
                     const double Sj = tot[0] * invZq;
+                    if (AN && scribe && lane == 0) TP.an[(long long)b * P.N + a].S[j] = Sj > RESIDUAL_FLOOR * w ? Sj : 0.0;
                     // A step whose mass is below 1e-13 of the weight before it counts as S = 0: P equals q, and what
                     // is left is the rounding of g.
                     if (Sj > RESIDUAL_FLOOR * w) {
@@ -610,6 +686,20 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     } else {
                         dead = true;       // S = 0 with w < 1: the weight drops to 0 (Traversal only)
                         w = 0.0;
+                    }
+                }
+
+                if (AN && scribe) {
+                    AnRec &Ar = TP.an[(long long)b * P.N + a];
+                    if (lane < kce) {
+                        const double q_t = eqx * invZq;
+                        Ar.A[kce][lane] = err ? 0.0 : (is_q ? q_t : ux / kappa);      // p_k(x_t)
+                        Ar.px[lane] = W.cpm[lane] / Z_p;
+                        Ar.qx[lane] = q_t;
+                    }
+                    if (lane == 0) {
+                        Ar.rho = an_rho; Ar.beta = an_beta; Ar.pacc = an_pacc; Ar.s_res = an_sres;
+                        Ar.k = kce; Ar.valid = err ? 0 : 1;
                     }
                 }
 

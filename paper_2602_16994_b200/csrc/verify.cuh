@@ -317,12 +317,20 @@ __device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk
     return adm;
 }
 
+// cross sums of the two rows for the Kullback-Leibler divergences (analysis instantiation only):
+// sum e_p x_p, sum e_p x_q, sum e_q x_p, sum e_q x_q with x = z s - O the exponents (a token cut from one row
+// has x = -inf there, which makes the divergence from the other row infinite, as it is)
+struct KlSums {
+    float pp, pq, qp, qq;
+};
+
 // One tile: wait for the stage, take the thread's 8 logits of both rows, hand the stage back, turn them
 // into e (EP, EQ), move dominant tokens to the list.  The thread's tail sums of e go to zs_p / zs_q.
-template <int DT, int NW>
+template <int DT, int NW, bool KLS = false>
 __device__ __forceinline__ void pass1_tile(const RingCtx &rc, int &stage, uint32_t &phase, bool &poisoned,
                                            const NodeRows &nr, int tile_index, int slot, int n_slice, int tid,
-                                           float (&EP)[8], float (&EQ)[8], WarpList &L, int &nl, float &zs_p, float &zs_q)
+                                           float (&EP)[8], float (&EQ)[8], WarpList &L, int &nl, float &zs_p, float &zs_q,
+                                           KlSums *kl = nullptr)
 {
     constexpr int NCONS = NW * 32;
     constexpr int TILE = NCONS * 8;
@@ -339,16 +347,36 @@ __device__ __forceinline__ void pass1_tile(const RingCtx &rc, int &stage, uint32
     if (++stage == rc.NS) { stage = 0; phase ^= 1u; }
     const int nvalid = poisoned ? 0 : n_slice - (tile_index * TILE + tid * 8);
     float z[8], dsx = 0.f;
-    unpack_chunk<DT>(raw_p, z);
-    mask_chunk(z, nvalid, nr.cut_p > -CUDART_INF_F, nr.cut_p);
-    float sum_p = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_p, EP, dsx), sum_q = 0.f;
-    if (nr.hq) {
+    float sum_p, sum_q = 0.f;
+    if (KLS) {
+        // the exponents themselves are needed: scalar form
+        float xp[8], xq[8];
+        unpack_chunk<DT>(raw_p, z);
+        mask_chunk(z, nvalid, nr.cut_p > -CUDART_INF_F, nr.cut_p);
+        sum_p = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { xp[k] = fmaf(z[k], nr.s_lo, fmaf(z[k], nr.s_hi, -(float)nr.O_p)); EP[k] = ex2_approx(xp[k]); sum_p += EP[k]; }
         unpack_chunk<DT>(raw_q, z);
         mask_chunk(z, nvalid, nr.cut_q > -CUDART_INF_F, nr.cut_q);
-        sum_q = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_q, EQ, dsx);
-    } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) EQ[k] = 0.f;
+        for (int k = 0; k < 8; ++k) { xq[k] = fmaf(z[k], nr.s_lo, fmaf(z[k], nr.s_hi, -(float)nr.O_q)); EQ[k] = ex2_approx(xq[k]); sum_q += EQ[k]; }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (EP[k] > 0.f) { kl->pp = fmaf(EP[k], xp[k], kl->pp); kl->pq = fmaf(EP[k], xq[k], kl->pq); }
+            if (EQ[k] > 0.f) { kl->qp = fmaf(EQ[k], xp[k], kl->qp); kl->qq = fmaf(EQ[k], xq[k], kl->qq); }
+        }
+    } else {
+        unpack_chunk<DT>(raw_p, z);
+        mask_chunk(z, nvalid, nr.cut_p > -CUDART_INF_F, nr.cut_p);
+        sum_p = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_p, EP, dsx);
+        if (nr.hq) {
+            unpack_chunk<DT>(raw_q, z);
+            mask_chunk(z, nvalid, nr.cut_q > -CUDART_INF_F, nr.cut_q);
+            sum_q = exp_chunk<false>(z, nr.s_hi, nr.s_lo, (float)nr.O_q, EQ, dsx);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) EQ[k] = 0.f;
+        }
     }
     // dominant tokens: a chunk whose sum stays below the threshold holds none (e >= 0)
     const bool room = nl < MW - MW_RES;
@@ -379,16 +407,16 @@ __device__ __forceinline__ void pass1_tile(const RingCtx &rc, int &stage, uint32
 // Pass 1 of a node.  es: [slot][p lo, p hi, q lo, q hi][NCONS] for the nsm shared-memory tiles; the last
 // nrg tiles of the slice stay in R.  On return nl is the fill of the warp's list and zs_p / zs_q the
 // thread's sums of the fp32 e it keeps (listed tokens excluded).
-template <int DT, int NW>
+template <int DT, int NW, bool KLS = false>
 __device__ __forceinline__ void pass1(const RingCtx &rc, int &stage, uint32_t &phase, bool &poisoned, const NodeRows &nr,
                                       float4 *es, int nsm, int nrg, int n_slice, int tid, Resident &R, WarpList &L,
-                                      int &nl, float &zs_p, float &zs_q)
+                                      int &nl, float &zs_p, float &zs_q, KlSums *kl = nullptr)
 {
     constexpr int NCONS = NW * 32;
     nl = 0; zs_p = 0.f; zs_q = 0.f;
     for (int i = 0; i < nsm; ++i) {
         float ep[8], eq[8];
-        pass1_tile<DT, NW>(rc, stage, phase, poisoned, nr, i, i, n_slice, tid, ep, eq, L, nl, zs_p, zs_q);
+        pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, i, i, n_slice, tid, ep, eq, L, nl, zs_p, zs_q, kl);
         float4 *d = es + (size_t)(i * 4) * NCONS + tid;
         d[0] = make_float4(ep[0], ep[1], ep[2], ep[3]);
         d[NCONS] = make_float4(ep[4], ep[5], ep[6], ep[7]);
@@ -398,7 +426,7 @@ __device__ __forceinline__ void pass1(const RingCtx &rc, int &stage, uint32_t &p
 #pragma unroll
     for (int j = 0; j < RT; ++j) {
         if (j < nrg) {
-            pass1_tile<DT, NW>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, R.p[j], R.q[j], L, nl, zs_p, zs_q);
+            pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, R.p[j], R.q[j], L, nl, zs_p, zs_q, kl);
         } else {
 #pragma unroll
             for (int k = 0; k < 8; ++k) { R.p[j][k] = 0.f; R.q[j][k] = 0.f; }
@@ -468,6 +496,33 @@ __device__ __forceinline__ double step_sweep(float4 *es, int nsm, int tid, Resid
         d += v;
     }
     return d;
+}
+
+// A read-only sweep over the thread's share of the resident node for the offline analysis: f.tail(e_p, e_q,
+// a0, a1) on every fp32 token (two running sums), f.exact(...) in fp64 on the entry of the warp's exact
+// list that falls to the lane.  Listed tokens are zero in the fp32 arrays; every f maps (0, 0) to nothing.
+template <int NW, typename F>
+__device__ __forceinline__ void reduce_sweep(const float4 *es, int nsm, int tid, const Resident &R, const WarpList &L,
+                                             int nl, const F &f, double &o0, double &o1)
+{
+    constexpr int NCONS = NW * 32;
+    float a0 = 0.f, a1 = 0.f;
+    for (int i = 0; i < nsm; ++i) {
+        float p[8], q[8];
+        const float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+        load_e8(d, NCONS, p);
+        load_e8(d + 2 * NCONS, NCONS, q);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) f.tail(p[k], q[k], a0, a1);
+    }
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) f.tail(R.p[j][k], R.q[j][k], a0, a1);
+    }
+    o0 = (double)a0;
+    o1 = (double)a1;
+    if ((tid & 31) < nl) f.exact(L.ep[tid & 31], L.eq[tid & 31], o0, o1);
 }
 
 // All-to-all of NV doubles per consumer warp of the cluster: tot[i] is the sum over every warp of every
