@@ -242,6 +242,17 @@ int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, 
  * benchmarks that report how many launches a timed region made).  Never fails. */
 int64_t spec_kernel_launches(void);
 
+/*
+ * Test hooks (no counterpart in the paper; not for production callers).  Every wait inside the kernels
+ * is bounded (Section "General rules": a wait that runs out is reported as SPEC_DEV_TIMEOUT, nothing
+ * hangs); these two settings let a test watch that happen.  wait_cycles: the limit of every on-device
+ * wait in clock cycles (<= 0: the default, about 2 s).  hold_slot: index b * N + node of one node whose
+ * Traversal weight the every-node kernel then never publishes, so that the node's own wait runs out
+ * (-1: none).  Synchronous (copies to constant memory of the current device); call it between
+ * verification calls, never while one is in flight.
+ */
+int32_t spec_test_hooks(int64_t wait_cycles, int32_t hold_slot);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,7 +27,7 @@ ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
            "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
            "spec_verify_specinfer_static", "spec_kernel_launches", "spec_analysis_workspace_bytes",
-           "spec_tree_analysis", "spec_latency_model")
+           "spec_tree_analysis", "spec_latency_model", "spec_test_hooks")
 
 
 class SpecIn(C.Structure):
@@ -99,6 +99,8 @@ def load_library(path: str = LIB_PATH):
     lib.spec_latency_model.restype = C.c_int32
     lib.spec_latency_model.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
+    lib.spec_test_hooks.restype = C.c_int32
+    lib.spec_test_hooks.argtypes = [C.c_int64, C.c_int32]
     _lib = lib
     return lib
 
@@ -120,6 +122,12 @@ def _ptr(t):
 def _stream_ptr(stream):
     s = stream if stream is not None else torch.cuda.current_stream()
     return C.c_void_p(s.cuda_stream)
+
+
+def set_test_hooks(wait_cycles: int = 0, hold_slot: int = -1):
+    """Test hooks: limit of the on-device waits in clock cycles (0: default) and one Traversal weight slot
+    (index b * N + node) that is left pending (-1: none)."""
+    _check(load_library().spec_test_hooks(int(wait_cycles), int(hold_slot)), "spec_test_hooks")
 
 
 def kernel_launches() -> int:

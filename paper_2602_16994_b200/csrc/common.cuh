@@ -10,7 +10,13 @@
 namespace specv {
 
 constexpr int KMAX = SPEC_MAX_CHILDREN;
-constexpr long long WAIT_CYCLES = 4000000000ll;   // every on-device wait gives up after about 2 s
+// Every on-device wait gives up after this many clock cycles (about 2 s).  A variable and not a constant so
+// that a test can shorten it (spec_test_hooks) and watch a wait run out without waiting for seconds.
+constexpr long long WAIT_CYCLES_DEFAULT = 4000000000ll;
+__constant__ long long c_wait_cycles = WAIT_CYCLES_DEFAULT;
+// Test hook: index b * N + node of a published-weight slot that the every-node kernel leaves pending (-1: none)
+__constant__ int c_hold_slot = -1;
+#define WAIT_CYCLES c_wait_cycles
 constexpr unsigned long long W_PENDING = 0xFFFFFFFFFFFFFFFFull;
 
 extern __shared__ __align__(128) unsigned char dyn_smem[];

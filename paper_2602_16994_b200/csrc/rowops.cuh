@@ -366,12 +366,13 @@ __global__ void __launch_bounds__(NT, 1) spec_probs_kernel(const TParams P)
     uint32_t tx = stage_row(ep, SL, P.dtype, row, tok0, n, &S.mbar, true);
     if (tid == 0 && tx) mbar_expect_tx(&S.mbar, tx);
     stage_row(ep, SL, P.dtype, row, tok0, n, &S.mbar, false);
-    if (tx) {
-        mbar_wait(&S.mbar, 0);
-    }
+    bool gave_up = false;
+    if (tx) gave_up = !mbar_wait(&S.mbar, 0);
     __syncthreads();
-    bool nan = false;
-    float m = warp_max(raw_max(ep, SL, P.dtype, n, nan));
+    bool nan = gave_up;          // a copy that was given up on: the row comes out as a non-finite one
+    bool nan2 = false;
+    float m = warp_max(raw_max(ep, SL, P.dtype, n, nan2));
+    nan = nan || nan2;
     if ((tid & 31) == 0) S.warp_part[tid >> 5][0] = (double)m;
     int any_nan = __syncthreads_or((int)nan);
     m = -CUDART_INF_F;
@@ -457,10 +458,12 @@ __global__ void __launch_bounds__(NT, 1) spec_bonus_kernel(const BParams P)
     uint32_t tx = stage_row(ep, SL, SPEC_F32, row, tok0, n, &S.mbar, true);
     if (tid == 0 && tx) mbar_expect_tx(&S.mbar, tx);
     stage_row(ep, SL, SPEC_F32, row, tok0, n, &S.mbar, false);
-    if (tx) {
-        mbar_wait(&S.mbar, 0);
-    }
+    int gave_up = 0;
+    if (tx) gave_up = mbar_wait(&S.mbar, 0) ? 0 : 1;
     for (int i = n + tid; i < SL; i += NT) ep[i] = 0.f;     // padding carries no weight
+    // a copy that was given up on: the slice counts as empty (its bytes may still be on their way)
+    if (__syncthreads_or(gave_up))
+        for (int i = tid; i < SL; i += NT) ep[i] = 0.f;
     __syncthreads();
     // slice total in the same order the search will use is not required: the search rescans
     double acc = 0.0;

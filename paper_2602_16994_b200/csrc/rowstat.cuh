@@ -285,11 +285,30 @@ __global__ void __launch_bounds__(NT, 2) spec_row_stat_kernel(const RParams P)
             } else {
                 for (int e = (int)(body / 4) + tid; e < n; e += NT) ((float *)raw)[e] = __ldg((const float *)src + e);
             }
+            int gave_up = 0;
             if (body) {
-                mbar_wait(&S.mbar, phase);
+                gave_up = mbar_wait(&S.mbar, phase) ? 0 : 1;
                 phase ^= 1u;
             }
-            __syncthreads();
+            // a copy that was given up on: the row is reported, not used (the decision is cluster-wide)
+            gave_up = __syncthreads_or(gave_up);
+            {
+                double v[4] = {(double)gave_up, 0.0, 0.0, 0.0};
+                cluster_allgather4(S, xpar, C, rank, v);
+                gave_up = 0;
+                for (int r = 0; r < C; ++r) gave_up |= S.xv[xpar][r][0] != 0.0;
+                xpar ^= 1;
+            }
+            if (gave_up) {
+                if (rank == 0 && tid == 0) {
+                    RowPart r = {};
+                    r.cut = -CUDART_INF_F; r.O = ROWPART_EMPTY; r.bad = ROW_TIMEOUT;
+                    *out = r;
+                    P.cut[row * 2 + which] = -CUDART_INF_F;
+                }
+                __syncthreads();
+                continue;
+            }
         }
         const float Tf = P.T_seq ? __ldg(P.T_seq + b) : P.T;
         const float sf = 1.4426950408889634f / Tf;

@@ -642,6 +642,18 @@ int32_t spec_query_plan(int32_t V, int32_t logits_dtype, int32_t *cluster_size, 
 
 int64_t spec_kernel_launches(void) { return (int64_t)g_kernel_launches.load(std::memory_order_relaxed); }
 
+int32_t spec_test_hooks(int64_t wait_cycles, int32_t hold_slot)
+{
+    const long long wc = wait_cycles > 0 ? (long long)wait_cycles : WAIT_CYCLES_DEFAULT;
+    const int hs = hold_slot;
+    if (cudaMemcpyToSymbol(c_wait_cycles, &wc, sizeof(wc)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_hold_slot, &hs, sizeof(hs)) != cudaSuccess) {
+        cudaGetLastError();
+        return SPEC_ERR_CUDA;
+    }
+    return SPEC_OK;
+}
+
 int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream)
 {
     return verify_common(in, out, ws, ws_bytes, stream, MODE_SPECINFER);

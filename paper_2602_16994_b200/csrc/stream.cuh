@@ -22,6 +22,7 @@ struct __align__(16) RowPart {
     int bad;           // 1: NaN or +inf seen; -1: row not read (draft row of a node without children)
 };
 constexpr int ROWPART_EMPTY = -(1 << 30);
+constexpr int ROW_TIMEOUT = 3;          // RowPart::bad of a row whose copy into shared memory was given up on
 
 namespace stream {
 

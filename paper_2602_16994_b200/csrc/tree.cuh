@@ -305,12 +305,13 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 int O_q = ROWPART_EMPTY;
                 float cut_q = -CUDART_INF_F;
                 bool bad = __ldcg(&rp[0].bad) != 0 || !(O_p > ROWPART_EMPTY) || !(Z_p > 0.0) || !(Z_p < CUDART_INF);
+                bool slow = __ldcg(&rp[0].bad) == ROW_TIMEOUT || (hq && __ldcg(&rp[1].bad) == ROW_TIMEOUT);
                 if (hq) {
                     Z_q = __ldcg(&rp[1].S); O_q = __ldcg(&rp[1].O); cut_q = __ldcg(&rp[1].cut);
                     bad = bad || __ldcg(&rp[1].bad) != 0 || !(O_q > ROWPART_EMPTY) || !(Z_q > 0.0) || !(Z_q < CUDART_INF);
                 }
                 err = __reduce_max_sync(0xffffffffu, err);
-                if (bad && !err) err = SPEC_DEV_NONFINITE;
+                if (bad && !err) err = slow ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE;
                 kind = (hint_dead || err) ? ITEM_DEAD : (hq ? ITEM_NODE : ITEM_LEAF);
                 __syncwarp();
                 if (kind == ITEM_NODE) {
@@ -421,7 +422,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     Rl.kappa = Zl; Rl.nsteps = 0;
                     Rl.cut_p = __ldcg(&rpl->cut); Rl.cut_q = -CUDART_INF_F;
                     Rl.next_child = -1;
-                    Rl.status = badl ? SPEC_DEV_NONFINITE : 0;
+                    Rl.status = badl ? (__ldcg(&rpl->bad) == ROW_TIMEOUT ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE) : 0;
                     Rl.bonus = -1; Rl.bonus_margin = 0.f;
                     Rl.w_in = trav ? thr_c : 1.0;
                     Rl.thr = thr_c;
@@ -644,8 +645,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                                 // the child polls the published slot only; the record is read after all of the
                                 // sequence's arrivals (each fenced), so no fence is needed between the two stores
                                 rec[cj].w_in = thr;
-                                *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
-                                    (unsigned long long)__double_as_longlong(thr);
+                                if (b * P.N + cj != c_hold_slot)      // (a test may ask for one slot to stay pending)
+                                    *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + cj) =
+                                        (unsigned long long)__double_as_longlong(thr);
                             } else {
                                 rec[cj].thr = thr;
                             }

@@ -207,7 +207,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spec_walk_kernel(const WP
                     const double Zr = __ldcg(&p->S);
                     const int Or = __ldcg(&p->O), bd = __ldcg(&p->bad);
                     // a row is not finite if it holds NaN / +inf, or no finite logit at all
-                    if (bd != -1 && (bd == 1 || !(Or > ROWPART_EMPTY) || !(Zr > 0.0) || !(Zr < CUDART_INF)))
+                    if (bd == ROW_TIMEOUT)
+                        st1 = max(st1, SPEC_DEV_TIMEOUT);
+                    else if (bd != -1 && (bd == 1 || !(Or > ROWPART_EMPTY) || !(Zr > 0.0) || !(Zr < CUDART_INF)))
                         st1 = max(st1, SPEC_DEV_NONFINITE);
                     S.t_Z[r2] = Zr; S.t_O[r2] = Or; S.t_cut[r2] = __ldcg(&p->cut);
                 }
