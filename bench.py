@@ -6,6 +6,9 @@ A step is one pass of the whole verification path over one batch of synthetic dr
 algorithm the workload lists (SpecInfer, Traversal Verification) is run once on the batch through
 the C-ABI library, logits already resident in HBM.  Consecutive calls use different input copies so
 that more than the L2 capacity is touched before a copy is read again (reads come from HBM).
+The timed block of K steps is repeated R times; the median block gives ``ms_per_step`` and ``value``,
+the fastest and slowest are reported beside it.  The row statistics kernel -- the one pass over the
+logits in HBM, the kernel the roofline is about -- is also timed by itself.
 One JSON line is printed by rank 0.
 
 ``--impl reference`` times the CPU checker (``oracle/``) on the host cores instead.
@@ -29,15 +32,13 @@ METRIC = "verified tree-nodes/sec"
 UNIT = "nodes/s"
 L2_BYTES = 132_644_864
 ROTATE_BYTES = 4 * L2_BYTES          # bytes touched before an input copy is read again
-# kernels of one call; the roofline figure is taken over the whole call (all of its kernels), so it
-# understates the fraction the streaming kernel reaches on its own
-KERNELS = {"specinfer": "spec_row_partial_kernel + spec_walk_kernel (whole specinfer call)",
-           "traversal": "spec_row_partial_kernel + spec_tree_kernel (whole traversal call)"}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (cold L2), for the kernels of a SpecInfer call on the headline workload: the row statistics
-# kernel (69.80 + 0.76 MB: every logit once) and the walk kernel (4.08 MB: the rows of the resident
-# nodes, which come from L2 in the benchmark).  Other workloads: not captured.
-TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_798_912 + 760_320 + 4_075_776}
+# The dominant kernel is the row statistics kernel: it is the only one that reads the logits from HBM
+# (every logit once), and both verifiers start with it.
+STAT_KERNEL = {False: "stream::spec_row_partial_kernel (row statistics: the one pass over the logits in HBM)",
+               True: "trunc::spec_row_trunc_kernel (+ rowstat::spec_row_stat_kernel for the rows it leaves over)"}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of that kernel from the ncu captures summarised
+# under profiles/ (cold L2).  Workloads without a capture: null.
+TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_798_912 + 760_320}
 
 
 def parse_args():
@@ -51,6 +52,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="enqueue every call from the host instead of replaying CUDA graphs")
+    ap.add_argument("--repeats", type=int, default=15, help="timed blocks of --steps steps (median reported)")
+    ap.add_argument("--gen", default="cpu", choices=["cpu", "cuda"],
+                    help="where the synthetic batches are drawn: cpu gives the same batch for a seed on every machine "
+                         "and on both arms; cuda is faster for the largest workloads")
     return ap.parse_args()
 
 
@@ -120,23 +125,37 @@ def oracle_step(oracle, host_arrays, w):
         (oracle.verify_specinfer if algo == "specinfer" else oracle.verify_traversal)(inp)
 
 
-def cpu_baseline(w, seconds: float) -> dict:
-    import oracle
-    from paper_2602_16994_b200 import synth
-    oracle.build()
-    host = synth.make_batch(w, seed=0, device="cpu").numpy()
-    oracle_step(oracle, host, w)                       # warm-up (page-in, thread pool)
+def _time_oracle(oracle, host, w, seconds: float):
+    """Passes of the checker over one batch for about ``seconds``: (passes, wall seconds)."""
     n, t0 = 0, time.perf_counter()
     while True:
         oracle_step(oracle, host, w)
         n += 1
         dt = time.perf_counter() - t0
         if dt >= seconds or n >= 10000:
-            break
-    nodes = n * w.draft_nodes() * len(w.algorithms)
-    return {"value": nodes / dt, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+            return n, dt
+
+
+def cpu_baseline(w, seconds: float) -> dict:
+    """The CPU checker as it stands on the host cores: all threads, then one thread, on the same batch."""
+    import oracle
+    from paper_2602_16994_b200 import synth
+    oracle.build()
+    host = synth.make_batch(w, seed=0, device="cpu").numpy()
+    cores = oracle.max_threads()
+    oracle_step(oracle, host, w)                       # warm-up (page-in, thread pool)
+    n, dt = _time_oracle(oracle, host, w, seconds)
+    nodes = w.draft_nodes() * len(w.algorithms)
+    oracle.set_threads(1)
+    try:
+        n1, dt1 = _time_oracle(oracle, host, w, seconds)
+    finally:
+        oracle.set_threads(cores)
+    return {"value": n * nodes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{n} passes over one {w.name} batch (B={w.B}, all algorithms), {dt:.1f} s of wall time; "
-                      "the checker evaluates only the nodes the walk reaches"}
+                      "the checker evaluates only the nodes the walk reaches",
+            "one_thread": {"value": n1 * nodes / dt1, "unit": UNIT, "cores": 1,
+                           "sample": f"{n1} passes over the same batch on one thread, {dt1:.1f} s of wall time"}}
 
 
 def run_reference(args):
@@ -193,7 +212,12 @@ def run_ours(args):
     bytes_per_call = w.logit_bytes()
     copies = max(2, min(24, -(-ROTATE_BYTES // bytes_per_call))) if bytes_per_call < ROTATE_BYTES else 1
     seeds = shard.rank_seeds(rank, world, copies)
-    batches = [synth.make_batch(w, seed=s, device=dev) for s in seeds]
+    # drawn by torch's CPU generator unless asked otherwise: a seed then names the same batch on every
+    # machine, and seed 0 (rank 0's first copy) is the batch the CPU checker legs run on
+    if args.gen == "cpu":
+        batches = [synth.make_batch(w, seed=s, device="cpu").to(dev) for s in seeds]
+    else:
+        batches = [synth.make_batch(w, seed=s, device=dev) for s in seeds]
     outs = binding.alloc_outputs(w.B, w.N, w.V, dev, features=w.features)
     stream = torch.cuda.current_stream()
     # arguments marshalled once per (algorithm, input copy); a call is then one C-ABI call
@@ -204,6 +228,9 @@ def run_ours(args):
     for a in w.algorithms:               # first calls set kernel attributes: they must not fall inside a capture
         for p in prepared[a]:
             p.launch(stream)
+    stat_prepared = prepared[w.algorithms[0]]
+    for p in stat_prepared:
+        p.launch_statistics_only(stream)
     torch.cuda.synchronize()
     launches_per_step = None
     if args.no_graph:
@@ -215,16 +242,22 @@ def run_ours(args):
         def step():
             for algo in w.algorithms:
                 call(algo)
+
+        def run_stats(n):
+            for i in range(n):
+                stat_prepared[i % len(batches)].launch_statistics_only(stream)
     else:
         # the library neither allocates nor synchronises, so a call can be captured: one graph per input
         # copy for the whole step, one per (algorithm, copy) for the per-algorithm figures
         side = torch.cuda.Stream()
 
-        def capture(algos, copies_):
+        def capture(algos, copies_, stats_only=False):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.stream(side):
                 with torch.cuda.graph(g, stream=side):
                     for i in copies_:
+                        if stats_only:
+                            stat_prepared[i].launch_statistics_only(side)
                         for a in algos:
                             prepared[a][i].launch(side)
             return g
@@ -238,6 +271,8 @@ def run_ours(args):
         round_graph = capture(w.algorithms, every)
         algo_round = {a: capture([a], every) for a in w.algorithms}
         algo_single = {a: [capture([a], [i]) for i in every] for a in w.algorithms}
+        stat_round = capture([], every, stats_only=True)
+        stat_single = [capture([], [i], stats_only=True) for i in every]
 
         def run_steps(n):
             for _ in range(n // len(batches)):
@@ -251,6 +286,12 @@ def run_ours(args):
             for i in range(n % len(batches)):
                 algo_single[algo][i].replay()
 
+        def run_stats(n):
+            for _ in range(n // len(batches)):
+                stat_round.replay()
+            for i in range(n % len(batches)):
+                stat_single[i].replay()
+
     if args.no_graph:
         def run_steps(n):
             for _ in range(n):
@@ -260,37 +301,65 @@ def run_ours(args):
             for _ in range(n):
                 call(algo)
 
+    def timed_blocks(run, n, repeats):
+        """``repeats`` blocks of ``n`` units each, timed on the device (barrier + synchronise on both sides of
+        every block, slowest rank counted): milliseconds per unit of every block."""
+        out = []
+        for _ in range(repeats):
+            shard.barrier(world)
+            torch.cuda.synchronize()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            run(n)
+            t1.record(stream)
+            torch.cuda.synchronize()
+            shard.barrier(world)
+            out.append(shard.max_over_ranks(t0.elapsed_time(t1), world, dev) / n)
+        return out
+
+    def spread(ms_list, scale=1.0):
+        return {"median": statistics.median(ms_list) * scale, "min": min(ms_list) * scale,
+                "max": max(ms_list) * scale, "blocks": len(ms_list)}
+
+    R = max(1, args.repeats)
     run_steps(max(3, args.warmup))
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    shard.barrier(world)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = binding.kernel_launches()
-    e0.record(stream)
-    run_steps(args.steps)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    # counted by the library at every launch site (for graphs: at capture, times the replays)
-    gpu_launches = (binding.kernel_launches() - launches0) if launches_per_step is None else launches_per_step * args.steps
-    shard.barrier(world)
-    ms_total = shard.max_over_ranks(e0.elapsed_time(e1), world, dev)
+    step_ms = timed_blocks(run_steps, args.steps, R)
+    # counted by the library at every launch site (for graphs: at capture, times the replays); per block
+    gpu_launches = ((binding.kernel_launches() - launches0) // R if launches_per_step is None
+                    else launches_per_step * args.steps)
     # per-algorithm call duration (the node kernel dominates a call), same rotation of cold inputs
     per_algo = {}
     for algo in w.algorithms:
         run_calls(algo, max(3, len(batches)))
-        torch.cuda.synchronize()
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a0.record(stream)
-        run_calls(algo, args.steps)
-        a1.record(stream)
-        torch.cuda.synchronize()
-        ms = a0.elapsed_time(a1) / args.steps
-        per_algo[algo] = {"us_per_call": ms * 1e3, "gbs": bytes_per_call / ms / 1e6,
-                          "nodes_per_s": w.draft_nodes() / ms * 1e3}
+        ms = timed_blocks(lambda n: run_calls(algo, n), args.steps, R)
+        med = statistics.median(ms)
+        per_algo[algo] = {"us_per_call": med * 1e3, "us_min": min(ms) * 1e3, "us_max": max(ms) * 1e3,
+                          "gbs": bytes_per_call / med / 1e6, "nodes_per_s": w.draft_nodes() / med * 1e3}
+    # the row statistics kernel by itself, same rotation of cold inputs
+    run_stats(max(3, len(batches)))
+    stat_ms = timed_blocks(run_stats, args.steps, R)
+    # the same calls on ONE input copy, read again and again: whatever of it fits in L2 comes from there
+    l2_warm = None
+    if copies > 1:
+        l2_warm = {}
+        for algo in w.algorithms:
+            if args.no_graph:
+                one = lambda n, a=algo: [prepared[a][0].launch(stream) for _ in range(n)]
+            else:
+                one = lambda n, a=algo: [algo_single[a][0].replay() for _ in range(n)]
+            one(3)
+            l2_warm[algo] = spread(timed_blocks(one, args.steps, max(3, R // 3)), 1e3)["median"]
+        one = ((lambda n: [stat_prepared[0].launch_statistics_only(stream) for _ in range(n)]) if args.no_graph
+               else (lambda n: [stat_single[0].replay() for _ in range(n)]))
+        one(3)
+        l2_warm["statistics_kernel"] = spread(timed_blocks(one, args.steps, max(3, R // 3)), 1e3)["median"]
+        l2_warm["unit"] = "us per call, one input copy re-read (it fits in L2): NOT an HBM figure"
     clocks = sampler.stop() if rank == 0 else None
     status_ok = bool((outs.status == 0).all().item())
 
@@ -332,13 +401,15 @@ def run_ours(args):
         peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     else:
         peak, peak_src = 6650.0, "fallback"
-    dom = w.algorithms[0]
-    achieved = per_algo[dom]["gbs"]
-    ms_per_step = ms_total / args.steps
+    trunc = (0 < w.top_k < w.V) or w.top_p < 1.0
+    stat_med = statistics.median(stat_ms)
+    achieved = bytes_per_call / stat_med / 1e6
+    ms_per_step = statistics.median(step_ms)
     nodes_per_step = w.draft_nodes() * len(w.algorithms)
     line = {
         "metric": METRIC, "value": world * nodes_per_step / ms_per_step * 1e3, "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+        "ms_per_step_spread": spread(step_ms), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": w.B, "N": w.N, "V": w.V, "logits": w.dtype,
                    "tree": f"delayed K={w.K} L1={w.L1} L2={w.L2}", "temperature": w.temperature, "top_k": w.top_k,
@@ -346,15 +417,24 @@ def run_ours(args):
                    "launch": "host enqueue per call" if args.no_graph else
                              f"CUDA graph replay: one graph holds a round of {len(batches)} steps (one per input copy), "
                              "single-step graphs for the remainder",
+                   "timing": f"{R} blocks of {args.steps} steps, each between two CUDA events on the launching stream; "
+                             "the median block is reported",
+                   "inputs": f"seeded, drawn on the {args.gen}",
                    "node_verifications_per_step": nodes_per_step, "logit_bytes_per_call": bytes_per_call,
                    "l2": f"{copies} input copies rotated ({copies * bytes_per_call / 1e6:.0f} MB touched between "
                          f"reuses, L2 is {L2_BYTES / 1e6:.0f} MB)" if copies > 1 else "inputs larger than L2"},
         "hbm_gbs": world * bytes_per_call * len(w.algorithms) / ms_per_step / 1e6,
         "per_algorithm": per_algo,
-        "roofline": {"bound": "hbm", "kernel": KERNELS[dom], "achieved": achieved, "peak": peak,
+        # the kernel that reads the logits from HBM, timed by itself; the fractions of whole calls (its
+        # bytes over the duration of statistics + node kernel) are given beside it
+        "roofline": {"bound": "hbm", "kernel": STAT_KERNEL[trunc], "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                     "frac_of_8TBs_nominal": achieved / 8000.0, "traffic": TRAFFIC_BYTES.get(w.name),
-                     "algorithmic_bytes_per_launch": bytes_per_call},
+                     "kernel_us": spread(stat_ms, 1e3),
+                     "frac_of_8TBs_nominal": achieved / 8000.0,
+                     "traffic": None if trunc else TRAFFIC_BYTES.get(w.name),
+                     "algorithmic_bytes_per_launch": bytes_per_call,
+                     "whole_call_frac": {a: per_algo[a]["gbs"] / peak for a in w.algorithms}},
+        "l2_warm_us": l2_warm,
         "clocks": clocks, "gpu_launches": gpu_launches,
         "status_ok": status_ok,
     }

@@ -122,6 +122,15 @@ int32_t spec_tree_probs(const SpecIn *in, int32_t which, float *probs, float *ro
                         void *ws, int64_t ws_bytes, void *stream);
 
 /*
+ * The first half of a verification call on its own: the statistics (reference, normaliser, top-k /
+ * top-p cut) of every row the verifiers read -- the one pass over the logits in HBM (Section 4's
+ * sampling transform, without materialising the distributions).  Results stay in `ws`; the entry point
+ * exists so that this pass can be timed and profiled by itself.  Same arguments and checks as the
+ * verifiers.
+ */
+int32_t spec_row_statistics(const SpecIn *in, void *ws, int64_t ws_bytes, void *stream);
+
+/*
  * SpecInfer verification (Algorithm 4 used top-down, Section 3.2 "OT-based algorithms"):
  * starting at the root, try the children of the current node in list order; child x is accepted
  * when u_accept < min(1, P(x)/q(x)), where P is the node's target distribution after the residual

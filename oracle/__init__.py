@@ -72,6 +72,8 @@ def lib():
         _lib.oracle_sample_bonus.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                              C.c_void_p, C.c_void_p]
         _lib.oracle_max_threads.restype = C.c_int32
+        _lib.oracle_set_threads.restype = None
+        _lib.oracle_set_threads.argtypes = [C.c_int32]
         _lib.oracle_spectr_rho.restype = C.c_double
         _lib.oracle_spectr_rho.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32]
         _lib.oracle_verify_otlp.restype = C.c_int32
@@ -101,6 +103,11 @@ def _ptr(a):
 
 def max_threads() -> int:
     return int(lib().oracle_max_threads())
+
+
+def set_threads(n: int) -> None:
+    """Threads the batch loops use from now on (timing only: results do not depend on it)."""
+    lib().oracle_set_threads(int(n))
 
 
 # ---------------------------------------------------------------------------------------------

@@ -703,3 +703,14 @@ int32_t oracle_max_threads(void)
     return 1;
 #endif
 }
+
+/* Number of threads the batch loops use from now on (n >= 1); arithmetic and results do not depend on it. */
+void oracle_set_threads(int32_t n)
+{
+#ifdef _OPENMP
+    extern void omp_set_num_threads(int);
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}

@@ -27,7 +27,7 @@ ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
            "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
            "spec_verify_specinfer_static", "spec_kernel_launches", "spec_analysis_workspace_bytes",
-           "spec_tree_analysis", "spec_latency_model", "spec_test_hooks")
+           "spec_tree_analysis", "spec_latency_model", "spec_test_hooks", "spec_row_statistics")
 
 
 class SpecIn(C.Structure):
@@ -99,6 +99,8 @@ def load_library(path: str = LIB_PATH):
     lib.spec_latency_model.restype = C.c_int32
     lib.spec_latency_model.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
+    lib.spec_row_statistics.restype = C.c_int32
+    lib.spec_row_statistics.argtypes = [C.POINTER(SpecIn), C.c_void_p, C.c_int64, C.c_void_p]
     lib.spec_test_hooks.restype = C.c_int32
     lib.spec_test_hooks.argtypes = [C.c_int64, C.c_int32]
     _lib = lib
@@ -326,6 +328,11 @@ class PreparedVerify:
         if rc != 0:
             _check(rc, "spec_verify_" + self.name)
         return self.outputs
+
+    def launch_statistics_only(self, stream=None):
+        """Only the row statistics pass of the call (``spec_row_statistics``), for timing it by itself."""
+        _check(self.lib.spec_row_statistics(self._in_ref, self.ws_ptr, self.ws_size, _stream_ptr(stream)),
+               "spec_row_statistics")
 
 
 @dataclass

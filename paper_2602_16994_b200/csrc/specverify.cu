@@ -654,6 +654,17 @@ int32_t spec_test_hooks(int64_t wait_cycles, int32_t hold_slot)
     return SPEC_OK;
 }
 
+int32_t spec_row_statistics(const SpecIn *in, void *ws, int64_t ws_bytes, void *stream)
+{
+    int rc = check_in(in, true);
+    if (rc) return rc;
+    const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
+    const WsLayout L = ws_layout(in);
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
+    SpecOut none = {};
+    return row_statistics(in, &none, (unsigned char *)ws, L, trunc, true, (cudaStream_t)stream, true);
+}
+
 int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream)
 {
     return verify_common(in, out, ws, ws_bytes, stream, MODE_SPECINFER);
