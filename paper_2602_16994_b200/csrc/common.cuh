@@ -79,6 +79,19 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
     return true;
 }
 
+// ---- programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
+// while the kernel before it still runs; it waits here before touching anything that kernel writes (a
+// no-op for a kernel launched without the attribute).  The earlier kernel lets its dependents be scheduled
+// with the second call; its memory is visible to them only after the wait.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- bulk asynchronous copy global -> shared, completing on an mbarrier (no multicast) -----------
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {

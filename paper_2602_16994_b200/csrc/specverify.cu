@@ -198,20 +198,25 @@ WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: on
 std::atomic<long long> g_kernel_launches{0};
 
 template <typename K>
-int launch_clustered(K kernel, int ctas, int C, int threads, int smem, cudaStream_t st, void *params_ptr)
+int launch_clustered(K kernel, int ctas, int C, int threads, int smem, cudaStream_t st, void *params_ptr,
+                     bool dependent = false)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas, 1, 1);
     cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = C;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // dependent: the kernel waits by itself (grid_dependency_wait) for the kernel before it in the stream, so
+    // its CTAs may be placed, and run their set-up, while that kernel's last CTAs still work
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = dependent ? 2 : 1;
     void *args[1] = {params_ptr};
     cudaError_t e = cudaLaunchKernelExC(&cfg, (const void *)kernel, args);
     if (e != cudaSuccess) { cudaGetLastError(); return SPEC_ERR_CUDA; }
@@ -375,7 +380,7 @@ int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
     int nc = resident_clusters(kernel, pl.C, threads, pl.smem);
     if (nc <= 0) return SPEC_ERR_UNSUPPORTED;
     if (nc > wp.B) nc = wp.B;
-    return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &wp);
+    return launch_clustered(kernel, nc * pl.C, pl.C, threads, pl.smem, st, &wp, true);
 }
 
 // Statistics of every row the verifiers read (reference, normaliser, cut; one record per row at the

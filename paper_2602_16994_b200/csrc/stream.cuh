@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
     const long long items = 2ll * P.B * P.N * P.NSL;
     const int slices_row = (P.V + SLICE - 1) / SLICE;
     const int slices_part = (slices_row + P.NSL - 1) / P.NSL;
+    grid_launch_dependents();     // a dependent verifier's CTAs may take the places of CTAs that have finished
 
     for (long long id = blockIdx.x; id < items; id += gridDim.x) {
         const int h = (int)(id % P.NSL);

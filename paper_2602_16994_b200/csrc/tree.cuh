@@ -62,7 +62,8 @@ struct __align__(16) NodeScalars {
     float cut_p, cut_q, u_a, ub_a;
     int kind, a, b, nsteps;
     unsigned leaf_mask;            // bit j: child j has no children
-    int pad[3];
+    int len;                       // FINISH item: the accepted path's length
+    int pad[2];
 };
 
 struct __align__(16) THdr {
@@ -234,6 +235,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 acc = __shfl_sync(0xffffffffu, acc, 0);
                 int err = 0;
                 if (acc == FIN_PENDING) { err = SPEC_DEV_TIMEOUT; S.poison = 1; }
+                const int len = acc >> FIN_LEN_SHIFT;
+                if (acc >= 0) acc &= (1 << FIN_LEN_SHIFT) - 1;
                 if (acc < 0 || err) {
                     kind = ITEM_IDLE;           // a faulty sequence has no bonus draw
                     if (lane == 0) { N.err = err; N.b = b; N.a = -1; }
@@ -247,7 +250,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         N.Z_p = __ldcg(&rc->Z_p); N.Z_q = __ldcg(&rc->Z_q);
                         N.O_p = (int)__ldcg(&rc->O_p); N.O_q = (int)__ldcg(&rc->O_q);
                         N.cut_p = __ldcg(&rc->cut_p); N.cut_q = __ldcg(&rc->cut_q);
-                        N.nsteps = nsteps; N.kc = hq ? 1 : 0; N.err = 0; N.a = a; N.b = b;
+                        N.nsteps = nsteps; N.kc = hq ? 1 : 0; N.err = 0; N.a = a; N.b = b; N.len = len;
                         N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
                     }
                 }
@@ -410,7 +413,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             int err = W.err;
             const int *parent = P.parent + (long long)b * P.topo_stride;
 
-            // a childless child is finished here, by the scribe warp: its record and its arrival
+            // a childless child is finished here, by the scribe warp: its record; its arrival is made with the node's
+            unsigned narr = 1u;
             auto finish_leaf = [&](int c, double thr_c) {
                 if (lane == 0) {
                     NodeRec &Rl = P.rec[(long long)b * P.N + c];
@@ -427,7 +431,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     Rl.w_in = trav ? thr_c : 1.0;
                     Rl.thr = thr_c;
                 }
-                arrive_sequence(P, b);
+                ++narr;
             };
 
             if (kind == ITEM_IDLE) {
@@ -487,24 +491,27 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                                 }
                             }
                         }
-                    arrive_sequence(P, b);
+                    arrive_sequence(P, b, narr);
                 }
-            } else if (kind == ITEM_NODE) {
-                NodeRows nr;
-                nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-                nr.s_hi = (float)nr.s_d;
-                if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
-                nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
-                if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
+            } else {
+              // ---- a node, or a sequence's FINISH item: pass 1 (one copy of its code for both): e = 2^(z s - O) of
+              // the rows, resident; dominant tokens to the exact lists ----------------------------------------------
+              NodeRows nr;
+              nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
+              nr.s_hi = (float)nr.s_d;
+              if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
+              nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
+              if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
+              // (a FINISH item reads the draft row only if the accepted node's state is not its target row)
+              nr.hq = kind == ITEM_NODE || W.nsteps != 0;
+              nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
+              set_list_thresholds(nr, W.Z_p, W.Z_q);
+              int nl;
+              float zs_p, zs_q;
+              KlSums kls = {0.f, 0.f, 0.f, 0.f};
+              pass1<DT, NW, AN>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q, &kls);
+              if (kind == ITEM_NODE) {
                 const int kc = W.kc;
-                nr.hq = true; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
-                set_list_thresholds(nr, W.Z_p, W.Z_q);
-
-                // ---- pass 1: e = 2^(z s - O) of both rows, resident; dominant tokens to the exact lists -------------
-                int nl;
-                float zs_p, zs_q;
-                KlSums kls = {0.f, 0.f, 0.f, 0.f};
-                pass1<DT, NW, AN>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q, &kls);
                 if (poisoned && !err) err = SPEC_DEV_TIMEOUT;
 
                 // ---- the rows' normalisers from what is resident (one exchange) -----------------------------------
@@ -720,23 +727,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         if (trav) { Rc.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) Rc.w_in = 1.0; }
                         else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
                     }
-                    arrive_sequence(P, b);
+                    arrive_sequence(P, b, narr);
                 }
-            } else {
+              } else {
                 // ---- FINISH: the accepted node back on chip, its recorded steps replayed, the bonus token drawn ---------
-                NodeRows nr;
-                nr.s_d = 1.4426950408889634 / (double)(P.T_seq ? __ldg(P.T_seq + b) : P.T);
-                nr.s_hi = (float)nr.s_d;
-                if ((double)nr.s_hi > nr.s_d) nr.s_hi = __uint_as_float(__float_as_uint(nr.s_hi) - 1u);
-                nr.s_lo = (float)(nr.s_d - (double)nr.s_hi);
-                if (!(nr.s_lo > 0.f)) nr.s_lo = 1.0e-30f;
                 const int nsteps = W.nsteps;
                 const bool is_q = nsteps == STATE_IS_Q;
-                nr.hq = nsteps != 0; nr.cut_p = W.cut_p; nr.cut_q = W.cut_q; nr.O_p = W.O_p; nr.O_q = W.O_q;
-                set_list_thresholds(nr, W.Z_p, W.Z_q);
-                int nl;
-                float zs_p, zs_q;
-                pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
                 double part = (double)zs_p + (lane < nl ? L.ep[lane] : 0.0);
                 if (is_q) part = (double)zs_q + (lane < nl ? L.eq[lane] : 0.0);
                 for (int j = 0; j < nsteps; ++j) part = step_sweep<NW>(es, nsm, tid, R, L, nl, W.cpm[j]);
@@ -762,7 +758,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     mg = (float)(bf.edge / tot[0]);
                 }
                 if (role == 1) {
-                    const int len = __ldcg(P.out.accept_len + b);
+                    const int len = W.len;
                     P.out.bonus_token[b] = tokn;
                     P.out.out_tokens[(long long)b * P.N + len] = tokn;
                     if (P.out.margin) P.out.margin[(long long)b * (P.N + 1) + P.N] = mg;
@@ -772,6 +768,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     int *ot = P.out.out_tokens + (long long)b * P.N;
                     for (int i = 0; i < P.N; ++i) ot[i] = -1;
                 }
+              }
             }
             // the scalars block may be rewritten
             __syncwarp();

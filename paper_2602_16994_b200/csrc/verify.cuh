@@ -54,6 +54,8 @@ constexpr int OMIN = -(1 << 30);
 constexpr int FAST_N = 32;   // trees up to this size are finished warp-parallel
 constexpr int FIN_PENDING = -1;     // VParams::fin of a sequence whose nodes are not all done
 constexpr int FIN_FAULTY = -2;      // ... of a sequence with a device-detected fault: no bonus draw
+constexpr int FIN_LEN_SHIFT = 12;   // a selected node is published as node | (accepted length << FIN_LEN_SHIFT)
+static_assert(SPEC_MAX_NODES <= (1 << FIN_LEN_SHIFT) && SPEC_MAX_NODES < (1 << (30 - FIN_LEN_SHIFT)), "packing of the published node");
 // A residual step whose mass is below this fraction of the mass before it is treated as S = 0: where P
 // equals q (the same row twice, two one-token nuclei on the same token) the exact difference is 0 and
 // the computed one a few 1e-16 of the mass (the rounding of the coefficient g).
@@ -255,14 +257,18 @@ struct NodeRows {
     float thrB_p, thrB_q;     // e above this: listed while the list has room (2^-DOM_B)
 };
 // Z: the row's normaliser from the statistics pass (fp32 exponentials: good enough for a threshold).
+// The second tier pays only where it can hold nearly all of a row's mass, that is on laws that are
+// peaked (near-greedy temperatures, short nuclei), and it is needed only where a residual mass is small
+// against the weight, which takes two laws that nearly agree on their heavy tokens: both rows peaked.
 // The largest e of a row lies in (1/2, 1], so Z > LIST_FLAT_Z means that no token holds more than
-// 1/LIST_FLAT_Z of the row's mass: on such a flat row the second tier would fill with arbitrary tokens
-// at once and buy nothing (small residual masses need two peaked laws), so it is left out.
-constexpr double LIST_FLAT_Z = 16.0;
+// 1/LIST_FLAT_Z of the row's mass.  On such a row the tier would fill with the first tokens it meets and
+// buy nothing, so it is left out; a node without a draft row (nothing is subtracted there) has no use
+// for it either.
+constexpr double LIST_FLAT_Z = 4.0;
 __device__ __forceinline__ void set_list_thresholds(NodeRows &nr, double Z_p, double Z_q)
 {
     const double a = 1.0 / (double)(1ull << DOM_A), b = 1.0 / (double)(1ull << DOM_B);
-    const bool flat = Z_p > LIST_FLAT_Z && (!nr.hq || Z_q > LIST_FLAT_Z);
+    const bool flat = !nr.hq || Z_p > LIST_FLAT_Z || Z_q > LIST_FLAT_Z;
     nr.thrA_p = (float)(Z_p * a);
     nr.thrB_p = flat ? nr.thrA_p : (float)(Z_p * b);
     nr.thrA_q = nr.hq ? (float)(Z_q * a) : CUDART_INF_F;
@@ -277,8 +283,8 @@ struct RingCtx {
 
 // Warp-collective: the tokens of this chunk position flagged in m_any (bit k: token k of the lane's
 // chunk; m_a: those above the always-listed threshold) are appended to the warp's list while it has
-// room, their exponentials evaluated in fp64 from the raw logits.  Returns the lane's mask of appended
-// tokens (the caller zeroes their fp32 copies).  n is the list's fill, the same in every lane.
+// room, as raw logits (pass1 evaluates the exponentials in fp64 once all tiles are in).  Returns the lane's
+// mask of appended tokens (the caller zeroes their fp32 copies).  n is the list's fill, the same in every lane.
 template <int DT>
 __device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk<DT> raw_p, const RawChunk<DT> raw_q,
                                              unsigned m_any, unsigned m_a, int nvalid, const NodeRows nr, int slot)
@@ -291,6 +297,8 @@ __device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk
     unsigned adm = 0;
 #pragma unroll 1
     for (int k = 0; k < 8; ++k) {
+        if (n >= MW - MW_RES) m_any &= m_a;           // no room left in the second tier
+        if (!__any_sync(0xffffffffu, (m_any >> k) != 0u)) break;
         const bool a = (m_a >> k) & 1u, b = ((m_any >> k) & 1u) && !a;
         const unsigned balA = __ballot_sync(0xffffffffu, a), balB = __ballot_sync(0xffffffffu, b);
         if (!(balA | balB)) continue;
@@ -306,9 +314,11 @@ __device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk
 #pragma unroll
             for (int kk = 1; kk < 8; ++kk)
                 if (kk == k) { z0 = zp[kk]; z1 = zq[kk]; }
+            // the raw logits for now (-inf: cut, or no draft row); pass1 turns every entry into its
+            // exponential at the end, all lanes at once, instead of one long fp64 chain per admission
             const bool valid = k < nvalid;
-            L.ep[idx] = (valid && z0 >= nr.cut_p) ? exp2_exact(z0, nr.s_d, nr.O_p) : 0.0;
-            L.eq[idx] = (valid && nr.hq && z1 >= nr.cut_q) ? exp2_exact(z1, nr.s_d, nr.O_q) : 0.0;
+            L.ep[idx] = (valid && z0 >= nr.cut_p) ? (double)z0 : -CUDART_INF;
+            L.eq[idx] = (valid && nr.hq && z1 >= nr.cut_q) ? (double)z1 : -CUDART_INF;
             L.pos[idx] = (slot << 8) | (lane << 3) | k;
             adm |= 1u << k;
         }
@@ -423,15 +433,34 @@ __device__ __forceinline__ void pass1(const RingCtx &rc, int &stage, uint32_t &p
         d[2 * NCONS] = make_float4(eq[0], eq[1], eq[2], eq[3]);
         d[3 * NCONS] = make_float4(eq[4], eq[5], eq[6], eq[7]);
     }
-#pragma unroll
+    // the register tiles: one copy of the tile's code (it is long, and the kernels are bound by instruction
+    // fetch as much as by anything else), its result moved to the tile's registers by predicated copies
+#pragma unroll 1
     for (int j = 0; j < RT; ++j) {
+        float ep[8], eq[8];
         if (j < nrg) {
-            pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, R.p[j], R.q[j], L, nl, zs_p, zs_q, kl);
+            pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, ep, eq, L, nl, zs_p, zs_q, kl);
         } else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) { R.p[j][k] = 0.f; R.q[j][k] = 0.f; }
+            for (int k = 0; k < 8; ++k) { ep[k] = 0.f; eq[k] = 0.f; }
+        }
+#pragma unroll
+        for (int jj = 0; jj < RT; ++jj) {
+            if (jj == j) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) { R.p[jj][k] = ep[k]; R.q[jj][k] = eq[k]; }
+            }
         }
     }
+    // the listed tokens' exponentials in fp64, entry `lane` (list_append left the raw logits)
+    __syncwarp();
+    if ((tid & 31) < nl) {
+        const int i = tid & 31;
+        const double zp = L.ep[i], zq = L.eq[i];
+        L.ep[i] = zp > -CUDART_INF ? exp2_exact((float)zp, nr.s_d, nr.O_p) : 0.0;
+        L.eq[i] = zq > -CUDART_INF ? exp2_exact((float)zq, nr.s_d, nr.O_q) : 0.0;
+    }
+    __syncwarp();
 }
 
 // hand a node's stages back unread (the node turned out not to need its rows)
@@ -718,9 +747,12 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
     for (int i = lane; i < N; i += 32) status = max(status, __ldcg(&rec[i].status));
     status = __reduce_max_sync(0xffffffffu, status);
     int acc = -1, len = 0;
+    const bool fast = N <= FAST_N;
+    // (a lane's own node: its parent and token, for the walks over the accepted path below)
+    const int par = fast && lane < N ? __ldg(parent + lane) : -2;
+    const int tok = fast && lane < N ? __ldg(token + lane) : -1;
     if (!status) {
-        if (N <= FAST_N) {
-            const int par = lane < N ? __ldg(parent + lane) : -2;
+        if (fast) {
             if (P.mode == MODE_SPECINFER) {
                 const int nx = lane < N ? __ldcg(&rec[lane].next_child) : -1;
                 acc = 0;
@@ -791,17 +823,36 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
     }
     if (status) { acc = -1; len = -1; }
     int *ot = P.out.out_tokens + (long long)b * N;
-    for (int i = lane; i < N; i += 32) ot[i] = -1;
-    __syncwarp();
+    if (fast) {
+        // position of the lane's node on the accepted path (1-based; 0: not on it), by walking up from the
+        // accepted node in registers; slot i of the output gets the token of the path's node at depth i + 1
+        int mine = 0, i = len;
+        for (int x = acc; x > 0 && i > 0; x = __shfl_sync(0xffffffffu, par, x), --i)
+            if (lane == x) mine = i;
+        for (int j = lane; j < N; j += 32) ot[j] = -1;
+        __syncwarp();
+        if (mine > 0) ot[mine - 1] = tok;
+    } else {
+        for (int i = lane; i < N; i += 32) ot[i] = -1;
+        __syncwarp();
+        if (lane == 0 && acc >= 0) {
+            int i = len;
+            for (int x = acc; x != 0 && i > 0; x = parent[x]) ot[--i] = token[x];
+        }
+    }
     if (lane == 0) {
         P.out.accepted_node[b] = acc;
         P.out.accept_len[b] = len;
         P.out.bonus_token[b] = -1;         // the FINISH item draws it
         P.out.status[b] = status;
-        if (acc >= 0) {
-            int i = len;
-            for (int x = acc; x != 0 && i > 0; x = parent[x]) ot[--i] = token[x];
-        }
+        if (P.out.margin) P.out.margin[(long long)b * (N + 1) + N] = CUDART_NAN_F;   // (the FINISH item's slot)
+    }
+    // publication: the outputs above are visible to whoever sees the accepted node (the diagnostics below
+    // are read by nobody on the device)
+    __syncwarp();
+    if (lane == 0) {
+        __threadfence();
+        *(volatile int *)(P.fin + b) = status ? FIN_FAULTY : (acc | (len << FIN_LEN_SHIFT));
     }
     if (P.out.node_thr)
         for (int i = lane; i < N; i += 32) P.out.node_thr[(long long)b * N + i] = (float)__ldcg(&rec[i].thr);
@@ -811,27 +862,20 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
         float *mg = P.out.margin + (long long)b * (N + 1);
         for (int i = lane; i < N; i += 32)
             mg[i] = i == 0 ? CUDART_NAN_F : (float)fabs((double)ua[i] - __ldcg(&rec[i].thr));
-        if (lane == 0) mg[N] = CUDART_NAN_F;
-    }
-    // publication: everything above is visible to whoever sees the accepted node
-    __syncwarp();
-    if (lane == 0) {
-        __threadfence();
-        *(volatile int *)(P.fin + b) = status ? FIN_FAULTY : acc;
     }
 }
 
-// One arrival of a node at its sequence, made by lane 0 of a converged warp; the warp that makes the
-// last of the N arrivals selects the accepted node.
-__device__ __forceinline__ void arrive_sequence(const VParams &P, int b)
+// The arrival of `count` nodes at their sequence (a node and the childless children it finished), made
+// by lane 0 of a converged warp; the warp that makes the last of the N arrivals selects the accepted node.
+__device__ __forceinline__ void arrive_sequence(const VParams &P, int b, unsigned count = 1u)
 {
     int last = 0;
     if ((threadIdx.x & 31) == 0) {
         // release: the node's record (written by this warp, ordered before by __syncwarp where another
         // lane wrote it) is visible to whoever sees the count; acquire: the last arrival sees all records
         unsigned prev;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(P.done + b), "r"(1u) : "memory");
-        last = (prev + 1u == (unsigned)P.N) ? 1 : 0;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(prev) : "l"(P.done + b), "r"(count) : "memory");
+        last = (prev + count == (unsigned)P.N) ? 1 : 0;
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) finalize_sequence(P, b);

@@ -98,6 +98,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spec_walk_kernel(const WP
     }
     __syncthreads();
     cluster_sync_all();
+    grid_dependency_wait();       // the row statistics come from the kernel before
 
     if (warp == NW) {
         // ======================= producer warp: loads the node the consumers ask for =====================
