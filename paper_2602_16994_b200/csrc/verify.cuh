@@ -433,23 +433,13 @@ __device__ __forceinline__ void pass1(const RingCtx &rc, int &stage, uint32_t &p
         d[2 * NCONS] = make_float4(eq[0], eq[1], eq[2], eq[3]);
         d[3 * NCONS] = make_float4(eq[4], eq[5], eq[6], eq[7]);
     }
-    // the register tiles: one copy of the tile's code (it is long, and the kernels are bound by instruction
-    // fetch as much as by anything else), its result moved to the tile's registers by predicated copies
-#pragma unroll 1
+#pragma unroll
     for (int j = 0; j < RT; ++j) {
-        float ep[8], eq[8];
         if (j < nrg) {
-            pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, ep, eq, L, nl, zs_p, zs_q, kl);
+            pass1_tile<DT, NW, KLS>(rc, stage, phase, poisoned, nr, nsm + j, SMT + j, n_slice, tid, R.p[j], R.q[j], L, nl, zs_p, zs_q, kl);
         } else {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) { ep[k] = 0.f; eq[k] = 0.f; }
-        }
-#pragma unroll
-        for (int jj = 0; jj < RT; ++jj) {
-            if (jj == j) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) { R.p[jj][k] = ep[k]; R.q[jj][k] = eq[k]; }
-            }
+            for (int k = 0; k < 8; ++k) { R.p[j][k] = 0.f; R.q[j][k] = 0.f; }
         }
     }
     // the listed tokens' exponentials in fp64, entry `lane` (list_append left the raw logits)
