@@ -281,16 +281,32 @@ struct RingCtx {
     int *poison;
 };
 
-// Warp-collective: the tokens of this chunk position flagged in m_any (bit k: token k of the lane's
-// chunk; m_a: those above the always-listed threshold) are appended to the warp's list while it has
-// room, as raw logits (pass1 evaluates the exponentials in fp64 once all tiles are in).  Returns the lane's
-// mask of appended tokens (the caller zeroes their fp32 copies).  n is the list's fill, the same in every lane.
+// the e of the 8 tokens a thread owns in one tile, both rows (passed by value to list_append)
+struct Chunk16 {
+    float p[8], q[8];
+};
+
+// Warp-collective, and out of line on purpose (it runs on a few per cent of the tiles, and the kernels
+// are short of instruction cache): the tokens of the lane's chunk whose e exceeds the always-listed
+// threshold (thrA), or the while-there-is-room threshold (tp, tq), are appended to the warp's list while
+// it has room, as raw logits (pass1 evaluates the exponentials in fp64 once all tiles are in).  n is the
+// list's fill, the same in every lane.  Returns (new fill << 8) | the lane's mask of appended tokens
+// (the caller zeroes their fp32 copies).
 template <int DT>
-__device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk<DT> raw_p, const RawChunk<DT> raw_q,
-                                             unsigned m_any, unsigned m_a, int nvalid, const NodeRows nr, int slot)
+__device__ __noinline__ unsigned list_append(WarpList &L, int n, const RawChunk<DT> raw_p, const RawChunk<DT> raw_q,
+                                             const Chunk16 e, float thrA_p, float thrA_q, float tp, float tq, int nvalid,
+                                             float cut_p, float cut_q, bool hq, int slot)
 {
     const int lane = threadIdx.x & 31;
     const unsigned lt = (1u << lane) - 1u;
+    unsigned m_any = 0, m_a = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const bool a = e.p[k] > thrA_p || e.q[k] > thrA_q;
+        const bool any = a || e.p[k] > tp || e.q[k] > tq;
+        m_any |= (any ? 1u : 0u) << k;
+        m_a |= (a ? 1u : 0u) << k;
+    }
     float zp[8], zq[8];
     unpack_chunk<DT>(raw_p, zp);
     unpack_chunk<DT>(raw_q, zq);
@@ -317,14 +333,14 @@ __device__ __noinline__ unsigned list_append(WarpList &L, int &n, const RawChunk
             // the raw logits for now (-inf: cut, or no draft row); pass1 turns every entry into its
             // exponential at the end, all lanes at once, instead of one long fp64 chain per admission
             const bool valid = k < nvalid;
-            L.ep[idx] = (valid && z0 >= nr.cut_p) ? (double)z0 : -CUDART_INF;
-            L.eq[idx] = (valid && nr.hq && z1 >= nr.cut_q) ? (double)z1 : -CUDART_INF;
+            L.ep[idx] = (valid && z0 >= cut_p) ? (double)z0 : -CUDART_INF;
+            L.eq[idx] = (valid && hq && z1 >= cut_q) ? (double)z1 : -CUDART_INF;
             L.pos[idx] = (slot << 8) | (lane << 3) | k;
             adm |= 1u << k;
         }
     }
     __syncwarp();
-    return adm;
+    return ((unsigned)n << 8) | adm;
 }
 
 // cross sums of the two rows for the Kullback-Leibler divergences (analysis instantiation only):
@@ -392,15 +408,13 @@ __device__ __forceinline__ void pass1_tile(const RingCtx &rc, int &stage, uint32
     const bool room = nl < MW - MW_RES;
     const float tp = room ? nr.thrB_p : nr.thrA_p, tq = room ? nr.thrB_q : nr.thrA_q;
     if (__any_sync(0xffffffffu, sum_p > tp || sum_q > tq)) {
-        unsigned m_any = 0, m_a = 0;
+        Chunk16 e;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const bool a = EP[k] > nr.thrA_p || EQ[k] > nr.thrA_q;
-            const bool any = a || EP[k] > tp || EQ[k] > tq;
-            m_any |= (any ? 1u : 0u) << k;
-            m_a |= (a ? 1u : 0u) << k;
-        }
-        const unsigned adm = list_append<DT>(L, nl, raw_p, raw_q, m_any, m_a, nvalid, nr, slot);
+        for (int k = 0; k < 8; ++k) { e.p[k] = EP[k]; e.q[k] = EQ[k]; }
+        const unsigned r = list_append<DT>(L, nl, raw_p, raw_q, e, nr.thrA_p, nr.thrA_q, tp, tq, nvalid, nr.cut_p,
+                                           nr.cut_q, nr.hq, slot);
+        nl = (int)(r >> 8);
+        const unsigned adm = r & 255u;
         if (adm) {
             sum_p = 0.f; sum_q = 0.f;
 #pragma unroll
@@ -733,18 +747,34 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
     const int *token = P.token + (long long)b * N;
     const NodeRec *rec = P.rec + (long long)b * N;
     const float *ua = P.u_accept + (long long)b * N;
+    int acc = -1, len = 0;
+    const bool fast = N <= FAST_N;
+    // a lane's own node, everything the selection needs of it fetched in one round of loads
+    const bool own = fast && lane < N;
+    const int par = own ? __ldg(parent + lane) : -2;
+    const int tok = own ? __ldg(token + lane) : -1;
+    const int nx = own ? __ldcg(&rec[lane].next_child) : -1;
+    const double thr_l = own ? __ldcg(&rec[lane].thr) : 0.0;
+    const float ua_l = own ? __ldg(ua + lane) : 0.f;
     int status = 0;
     for (int i = lane; i < N; i += 32) status = max(status, __ldcg(&rec[i].status));
     status = __reduce_max_sync(0xffffffffu, status);
-    int acc = -1, len = 0;
-    const bool fast = N <= FAST_N;
-    // (a lane's own node: its parent and token, for the walks over the accepted path below)
-    const int par = fast && lane < N ? __ldg(parent + lane) : -2;
-    const int tok = fast && lane < N ? __ldg(token + lane) : -1;
+    // (fast path) the ancestors of the lane's node, itself included, as a bit mask: pointer doubling, five
+    // rounds for up to 32 levels; on a tree whose parents come first (checked by the nodes: status)
+    unsigned anc = own ? 1u << lane : 0u;
+    if (fast) {
+        int jump = own ? par : -1;
+#pragma unroll
+        for (int it = 0; it < 5; ++it) {
+            const int src = jump < 0 ? lane : jump;
+            const unsigned up = __shfl_sync(0xffffffffu, anc, src);
+            const int jj = __shfl_sync(0xffffffffu, jump, src);
+            if (jump >= 0) { anc |= up; jump = jj; }
+        }
+    }
     if (!status) {
         if (fast) {
             if (P.mode == MODE_SPECINFER) {
-                const int nx = lane < N ? __ldcg(&rec[lane].next_child) : -1;
                 acc = 0;
                 for (int hop = 0; hop < N; ++hop) {
                     const int n = __shfl_sync(0xffffffffu, nx, acc);
@@ -752,27 +782,21 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
                     acc = n;
                 }
             } else {
-                // depth-first post-order; the first node with u < w_fin (the root always) is accepted
-                const bool hit = lane < N && (lane == 0 || (double)__ldg(ua + lane) < __ldcg(&rec[lane].thr));
+                // Depth-first post-order; the first node with u < w_fin (the root always) is accepted.  With H the
+                // set of nodes whose subtree holds such a node: from the root, step to the first child in H
+                // while there is one (the subtrees of the children before it are rejected as a whole).
+                const bool hit = own && (lane == 0 || (double)ua_l < thr_l);
+                const unsigned H = __reduce_or_sync(0xffffffffu, hit ? anc : 0u);
                 int cur = 0;
-                for (int guard = 0; guard < 4 * N + 4 && acc < 0; ++guard) {
-                    for (;;) {
-                        const unsigned m = __ballot_sync(0xffffffffu, par == cur);
-                        if (!m) break;
-                        cur = __ffs(m) - 1;
-                    }
-                    for (;;) {
-                        const int h = __shfl_sync(0xffffffffu, (int)hit, cur);
-                        if (cur == 0 || h) { acc = cur; break; }
-                        const int p = __shfl_sync(0xffffffffu, par, cur);
-                        const unsigned m = __ballot_sync(0xffffffffu, par == p) & ~((2u << cur) - 1u);
-                        if (m) { cur = __ffs(m) - 1; break; }
-                        cur = p;
-                    }
+                for (int d = 0; d < N; ++d) {
+                    const unsigned m = __ballot_sync(0xffffffffu, own && par == cur && ((H >> lane) & 1u));
+                    if (!m) break;
+                    cur = __ffs(m) - 1;
                 }
+                acc = cur;
             }
-            if (acc >= 0)
-                for (int x = acc; x > 0 && len <= N; x = __shfl_sync(0xffffffffu, par, x)) ++len;
+            // the path's length is the accepted node's depth
+            len = __popc(__shfl_sync(0xffffffffu, anc, acc)) - 1;
         } else {
             if (lane == 0) {
                 if (P.mode == MODE_SPECINFER) {
@@ -814,11 +838,10 @@ __device__ __noinline__ void finalize_sequence(const VParams &P, int b)
     if (status) { acc = -1; len = -1; }
     int *ot = P.out.out_tokens + (long long)b * N;
     if (fast) {
-        // position of the lane's node on the accepted path (1-based; 0: not on it), by walking up from the
-        // accepted node in registers; slot i of the output gets the token of the path's node at depth i + 1
-        int mine = 0, i = len;
-        for (int x = acc; x > 0 && i > 0; x = __shfl_sync(0xffffffffu, par, x), --i)
-            if (lane == x) mine = i;
+        // a node on the accepted path (an ancestor of the accepted node, or that node; not the root) puts its
+        // token at its depth - 1
+        const unsigned path = acc >= 0 ? __shfl_sync(0xffffffffu, anc, acc) : 0u;
+        const int mine = (own && lane > 0 && ((path >> lane) & 1u)) ? __popc(anc) - 1 : 0;
         for (int j = lane; j < N; j += 32) ot[j] = -1;
         __syncwarp();
         if (mine > 0) ot[mine - 1] = tok;
