@@ -171,7 +171,7 @@ inline int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
 
 // workspace layout: node records | published weights + arrival counters (cleared per call) | row cuts
 struct WsLayout {
-    int64_t rec, pub, fin, done, ticket, cut, todo, stat, gseq, total;
+    int64_t rec, pub, fin, best, done, ticket, order, cut, todo, stat, gseq, total;
 };
 constexpr int MAX_PARTS = 4;      // parts a row may be split into by the streaming statistics kernel
 WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: one record per row only
@@ -180,11 +180,15 @@ WsLayout ws_layout(const SpecIn *in, int slices = MAX_PARTS)   // slices = 0: on
     const int64_t nodes = (int64_t)in->B * in->N;
     int64_t o = 0;
     L.rec = o; o += up256(nodes * (int64_t)sizeof(NodeRec));
-    // set to all-ones per call: published weights, accepted nodes; set to zero: arrival counters, item counter
+    // set to all-ones per call: published weights, accepted nodes, earliest known acceptance; set to zero:
+    // arrival counters, item counter, post-order table
     L.pub = o; o += nodes * 8;
     L.fin = o; o += (int64_t)in->B * 4;
+    L.best = o; o += (int64_t)in->B * 4;
     L.done = o; o += (int64_t)in->B * 4;
     L.ticket = o; o += 4;
+    o = (o + 7) / 8 * 8;
+    L.order = o; o += nodes * 8;
     o = up256(o);
     L.cut = o; o += up256(nodes * 8);
     L.todo = o; o += up256(4 + nodes * 8);          // count, then ids of the rows left to the general top-k / top-p kernel
@@ -395,7 +399,7 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
     if (trunc) {
         if (init_nodes &&
             (cudaMemsetAsync(w + L.pub, 0xFF, (size_t)(L.done - L.pub), st) != cudaSuccess ||
-             cudaMemsetAsync(w + L.done, 0, (size_t)in->B * 4 + 4, st) != cudaSuccess)) {
+             cudaMemsetAsync(w + L.done, 0, (size_t)(L.order - L.done) + (size_t)in->B * in->N * 8, st) != cudaSuccess)) {
             cudaGetLastError();
             return SPEC_ERR_CUDA;
         }
@@ -419,6 +423,7 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
         if (init_nodes) {
             sp.w_pub = (unsigned long long *)(w + L.pub); sp.done = (unsigned int *)(w + L.done);
             sp.fin = (int *)(w + L.fin); sp.ticket = (unsigned int *)(w + L.ticket);
+            sp.best = (unsigned int *)(w + L.best); sp.order = (unsigned long long *)(w + L.order);
         }
         const long long items = 2ll * in->B * in->N * NSL;
         const unsigned grid = (unsigned)(items < (1ll << 20) ? items : (1ll << 20));
@@ -490,6 +495,11 @@ void fill_tparams(const SpecIn *in, const SpecOut *out, unsigned char *w, const 
     vp.w_pub = (unsigned long long *)(w + L.pub);
     vp.done = (unsigned int *)(w + L.done);
     vp.fin = (int *)(w + L.fin);
+    vp.best = (unsigned int *)(w + L.best);
+    vp.order = (unsigned long long *)(w + L.order);
+    // Traversal without per-node diagnostics: subtrees that come after a known acceptance in the traversal
+    // order are not evaluated
+    vp.prune = (mode == MODE_TRAVERSAL && !out->node_thr && !out->node_w_in && !out->margin) ? 1 : 0;
     vp.out = *out;
     tp.part = (const RowPart *)(w + L.stat);
     tp.gseq = (double *)(w + L.gseq);

@@ -44,6 +44,8 @@ struct SParams {
     unsigned long long *w_pub;   // [B*N]
     unsigned int *done;          // [B]
     int *fin;                    // [B] set to -1 (no accepted node selected yet)
+    unsigned int *best;          // [B] set to all-ones (no acceptance known yet)
+    unsigned long long *order;   // [B*N] set to 0 (post-order table not computed yet)
     unsigned int *ticket;        // [1] item counter of the every-node kernel
 };
 
@@ -101,7 +103,8 @@ __global__ void __launch_bounds__(NT, 2) spec_row_partial_kernel(const SParams P
         RowPart *out = P.part + row2 * P.NSL + h;
         if (P.w_pub && which == 0 && h == 0 && tid == 0) {
             P.w_pub[row] = W_PENDING;
-            if (a == 0) { P.done[b] = 0u; P.fin[b] = -1; }
+            P.order[row] = 0ull;
+            if (a == 0) { P.done[b] = 0u; P.fin[b] = -1; P.best[b] = 0xFFFFFFFFu; }
             if (row == 0) *P.ticket = 0u;
         }
         if (which == 1) {

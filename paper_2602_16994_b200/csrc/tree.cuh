@@ -63,7 +63,9 @@ struct __align__(16) NodeScalars {
     int kind, a, b, nsteps;
     unsigned leaf_mask;            // bit j: child j has no children
     int len;                       // FINISH item: the accepted path's length
-    int pad[2];
+    int pruned;                    // the node lies wholly after a known acceptance: weight 0 without waiting for it
+    unsigned ord_a;                // the node's entry of the post-order table (0: not known)
+    unsigned cord[KMAX];           // ... and its children's
 };
 
 struct __align__(16) THdr {
@@ -92,6 +94,46 @@ __device__ __forceinline__ void mbar_arrive_remote(uint64_t *bar, uint32_t rank)
         "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(smem_u32(bar)), "r"(rank)
         : "memory");
 }
+// Entry `lane` of the post-order table of one tree of at most 32 nodes (children visited in index order, a
+// node after its subtree: the order in which Traversal Verification tests the nodes).  Low word:
+// 0x80000000 | rank << 8 | F, with F the number of nodes that come wholly before the node's subtree; high word:
+// the node's ancestors, itself included, as a bit mask.  0 for every node of a tree whose parents do not come first.  From ancestor masks: F(v) sums, over v and its
+// ancestors, the sizes of the subtrees of their earlier siblings, and rank(v) = F(v) + size(v) - 1.
+__device__ __noinline__ unsigned long long post_order_entry(const int *parent, int N, int lane)
+{
+    const bool own = lane < N;
+    const int par = own ? __ldg(parent + lane) : -2;
+    if (__any_sync(0xffffffffu, own && (lane == 0 ? par != -1 : (par < 0 || par >= lane)))) return 0ull;
+    unsigned anc = own ? 1u << lane : 0u;
+    int jump = own ? par : -1;
+#pragma unroll
+    for (int it = 0; it < 5; ++it) {
+        const int src = jump < 0 ? lane : jump;
+        const unsigned up = __shfl_sync(0xffffffffu, anc, src);
+        const int jj = __shfl_sync(0xffffffffu, jump, src);
+        if (jump >= 0) { anc |= up; jump = jj; }
+    }
+    unsigned D = 0;                 // the node's subtree: the lanes whose ancestor mask holds it
+    for (int v = 0; v < N; ++v) {
+        const unsigned m = __ballot_sync(0xffffffffu, (anc >> v) & 1u);
+        if (lane == v) D = m;
+    }
+    unsigned Em = 0;                // the subtrees of the node's earlier siblings
+    for (int sb = 1; sb < N; ++sb) {
+        const unsigned Ds = __shfl_sync(0xffffffffu, D, sb);
+        const int ps = __shfl_sync(0xffffffffu, par, sb);
+        if (own && sb < lane && ps == par) Em |= Ds;
+    }
+    const int E = __popc(Em);
+    int F = 0;
+    for (int x = 1; x < N; ++x) {
+        const int Ex = __shfl_sync(0xffffffffu, E, x);
+        if ((anc >> x) & 1u) F += Ex;
+    }
+    const int rank = F + __popc(D) - 1;
+    return own ? (((unsigned long long)anc << 32) | 0x80000000u | ((unsigned)rank << 8) | (unsigned)F) : 0ull;
+}
+
 // bounded poll of a published weight; W_PENDING when the limit ran out
 __device__ __forceinline__ unsigned long long poll_weight(const unsigned long long *slot_, const int *poison)
 {
@@ -156,22 +198,44 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
         bool ok = true;
         for (int kidx = 0; ok; ++kidx) {
             const int buf = kidx & 1;
+            // once its first item is under way, one producer of the cluster writes the post-order tables of its
+            // share of the sequences (a hint for the item hand-out below: absent entries only mean no skipping)
+            if (kidx == 1 && trav && P.N <= 32 && rank == (unsigned)(C > 1 ? 1 : 0)) {
+                const int ncl = (int)(gridDim.x / (unsigned)C);
+                for (int bb = (int)(blockIdx.x / (unsigned)C); bb < P.B; bb += ncl) {
+                    const unsigned long long e = post_order_entry(P.parent + (long long)bb * P.topo_stride, P.N, lane);
+                    if (lane < P.N) *(volatile unsigned long long *)(P.order + (long long)bb * P.N + lane) = e;
+                }
+            }
             // ---- the item: drawn by the first CTA's producer, passed on to the others ---------------------------
             if (rank == 0) {
                 unsigned long long val = 0;
                 int w = 1;
+                unsigned t = 0;
                 if (lane == 0) {
                     // every producer has read the item that used this slot before
                     if (kidx >= 2) w = mbar_wait_cluster(&S.abar[buf], (uint32_t)(((kidx >> 1) - 1) & 1)) ? 1 : 0;
-                    const unsigned t = atomicAdd(TP.ticket, 1u);
-                    unsigned hint = 0;
-                    if (trav && (long long)t < total && t >= (unsigned)P.B) {
-                        // a node whose weight is already known to be 0 needs no rows
-                        const int a = (int)(t / (unsigned)P.B), b = (int)(t % (unsigned)P.B);
-                        if (*(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + a) == 0ull) hint = 1;
-                    }
-                    val = (unsigned long long)t | ((unsigned long long)hint << 32);
+                    t = atomicAdd(TP.ticket, 1u);
                 }
+                t = __shfl_sync(0xffffffffu, t, 0);
+                unsigned hint = 0;
+                if (trav && (long long)t < total && t >= (unsigned)P.B) {
+                    const int a = (int)(t / (unsigned)P.B), b = (int)(t % (unsigned)P.B);
+                    // A node whose weight is already known to be 0 needs no rows, and the weight is 0 as soon as
+                    // an ancestor's is (one load per lane: the weights of the tree's first 32 nodes).  Neither
+                    // does a subtree that comes wholly after a node known to be accepted.
+                    const unsigned long long e = *(volatile unsigned long long *)(P.order + (long long)b * P.N + a);
+                    const unsigned ord = (unsigned)e;
+                    unsigned anc = (ord >> 31) ? (unsigned)(e >> 32) : 0u;
+                    if (a < 32) anc |= 1u << a;
+                    const bool zero = lane < P.N && ((anc >> lane) & 1u) &&
+                                      *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + lane) == 0ull;
+                    const unsigned zm = __ballot_sync(0xffffffffu, zero);
+                    if (zm) hint = (zm >> (a < 32 ? a : 0)) & 1u ? 1 : 3;
+                    if (a >= 32 && *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + a) == 0ull) hint = 1;
+                    if (P.prune && (ord >> 31) && *(volatile unsigned *)(P.best + b) < (ord & 255u)) hint = 2;
+                }
+                val = (unsigned long long)t | ((unsigned long long)hint << 32);
                 w = __shfl_sync(0xffffffffu, w, 0);
                 val = __shfl_sync(0xffffffffu, val, 0);
                 if (!w) { S.poison = 1; val = 0xFFFFFFFFull; }       // gave up: everybody leaves
@@ -191,7 +255,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 if (!w) { S.poison = 1; item = 0xFFFFFFFFull; }
             }
             const long long t = (long long)(item & 0xFFFFFFFFull);
-            const bool hint_dead = (item >> 32) != 0;
+            // (1: its own weight is 0; 2, 3: wholly after an accepted node, or below a node of weight 0 -- its weight
+            // is, or may as well be, 0, and is not waited for)
+            const bool hint_dead = (item >> 32) != 0, hint_pruned = (item >> 32) >= 2;
 
             // a childless node other than the root is finished by its parent: its ticket is skipped by everybody
             // (one whose parent index is not valid is nobody's child: it stays an item and reports the fault)
@@ -269,6 +335,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
                     }
                     N.u_a = __ldg(P.u_accept + (long long)b * P.N + a);
+                    N.pruned = hint_pruned ? 1 : 0;
+                    N.ord_a = P.prune ? (unsigned)*(volatile unsigned long long *)(P.order + (long long)b * P.N + a) : 0u;
                     N.ub_a = __ldg(P.u_bonus + (long long)b * P.N + a);
                     N.a = a; N.b = b; N.nsteps = 0;
                 }
@@ -281,6 +349,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         if (pos < KMAX) {
                             const int x = __ldg(token + c);
                             N.child[pos] = c;
+                            N.cord[pos] = P.prune ? (unsigned)*(volatile unsigned long long *)(P.order + (long long)b * P.N + c) : 0u;
                             N.cu[pos] = __ldg(P.u_accept + (long long)b * P.N + c);
                             N.cpm[pos] = (double)x;          // parked here until the exponentials are known
                             if (x < 0 || x >= P.V) err = SPEC_DEV_TOKEN;
@@ -415,7 +484,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
 
             // a childless child is finished here, by the scribe warp: its record; its arrival is made with the node's
             unsigned narr = 1u;
-            auto finish_leaf = [&](int c, double thr_c) {
+            auto finish_leaf = [&](int c, double thr_c, int j = -1) {
                 if (lane == 0) {
                     NodeRec &Rl = P.rec[(long long)b * P.N + c];
                     const RowPart *rpl = TP.part + ((long long)b * P.N + c) * 2;
@@ -430,6 +499,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     Rl.bonus = -1; Rl.bonus_margin = 0.f;
                     Rl.w_in = trav ? thr_c : 1.0;
                     Rl.thr = thr_c;
+                    // accepted if reached: nothing that comes after it in the traversal order matters any more
+                    if (P.prune && j >= 0 && (W.cord[j] >> 31) && (double)W.cu[j] < thr_c)
+                        atomicMin(P.best + b, (W.cord[j] >> 8) & 255u);
                 }
                 ++narr;
             };
@@ -442,7 +514,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 // weight 0 (or under a faulty node) can be accepted -----------------------------------------------
                 if (scribe) {
                     double w_in = 1.0;
-                    if (trav && a > 0 && !err) {
+                    if (W.pruned) {
+                        w_in = 0.0;        // whatever its weight, it cannot be the accepted node
+                    } else if (trav && a > 0 && !err) {
                         unsigned long long bits = W_PENDING;
                         if (lane == 0) bits = poll_weight(P.w_pub + (long long)b * P.N + a, &S.poison);
                         bits = __shfl_sync(0xffffffffu, bits, 0);
@@ -645,7 +719,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                     if (scribe) {
                         const int cj = W.child[j];
                         if ((W.leaf_mask >> j) & 1u) {
-                            finish_leaf(cj, thr);
+                            finish_leaf(cj, thr, j);
                         } else if (lane == 0) {
                             NodeRec *rec = P.rec + (long long)b * P.N;
                             if (trav) {
@@ -726,6 +800,8 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                         Rc.bonus = -1; Rc.bonus_margin = 0.f;
                         if (trav) { Rc.thr = (a == 0) ? 1.0 : w_fin; if (a == 0) Rc.w_in = 1.0; }
                         else { Rc.w_in = 1.0; if (a == 0) Rc.thr = 1.0; }
+                        if (P.prune && a > 0 && !err && (W.ord_a >> 31) && (double)W.u_a < w_fin)
+                            atomicMin(P.best + b, (W.ord_a >> 8) & 255u);
                     }
                     arrive_sequence(P, b, narr);
                 }

@@ -88,6 +88,10 @@ struct VParams {
     unsigned long long *w_pub;   // [B*N] weight handed to a node by its parent (Traversal), W_PENDING until known
     unsigned int *done;          // [B] arrivals per sequence (one per node); the last one selects the accepted node
     int *fin;                    // [B] the accepted node once it is selected (FIN_PENDING before, FIN_FAULTY for a faulty sequence)
+    unsigned int *best;          // [B] smallest post-order rank of a node known to be accepted if reached (all-ones: none)
+    unsigned long long *order;   // [B*N] low word: 0x80000000 | post-order rank << 8 | nodes wholly before the node's
+                                 // subtree; high word: the node's ancestors (itself included) as a bit mask; 0: not computed
+    int prune;                   // Traversal: skip subtrees that lie wholly after a known acceptance
     SpecOut out;
 };
 
