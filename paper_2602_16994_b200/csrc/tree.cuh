@@ -73,6 +73,7 @@ struct __align__(16) THdr {
     unsigned long long item[2];    // ticket | (weight already 0) << 32, written by the first CTA's producer
     double wtile[NWMAX + 1][TMAX];
     NodeScalars sc[2];
+    NodeScalars scd;               // the producer's own block for a node it finishes by itself (weight known to be 0)
     int poison;
 };
 
@@ -132,6 +133,60 @@ __device__ __noinline__ unsigned long long post_order_entry(const int *parent, i
     }
     const int rank = F + __popc(D) - 1;
     return own ? (((unsigned long long)anc << 32) | 0x80000000u | ((unsigned)rank << 8) | (unsigned)F) : 0ull;
+}
+
+// The record of a childless node c of sequence b, finished by whoever hands it its weight thr_c (lane 0 of a
+// converged warp writes; the node's arrival is counted by the caller).  Accepted if reached (Traversal without
+// diagnostics, `ord` its post-order entry, u its uniform): nothing after it in the traversal order matters.
+__device__ __noinline__ void leaf_record(const VParams &P, const RowPart *part, int b, int c, double thr_c, unsigned ord,
+                                         float u)
+{
+    if ((threadIdx.x & 31) != 0) return;
+    const bool trav = P.mode == MODE_TRAVERSAL;
+    NodeRec &Rl = P.rec[(long long)b * P.N + c];
+    const RowPart *rpl = part + ((long long)b * P.N + c) * 2;
+    const double Zl = __ldcg(&rpl->S);
+    const int Ol = __ldcg(&rpl->O);
+    const bool badl = __ldcg(&rpl->bad) != 0 || !(Ol > ROWPART_EMPTY) || !(Zl > 0.0) || !(Zl < CUDART_INF);
+    Rl.O_p = (double)Ol; Rl.Z_p = Zl; Rl.O_q = 0.0; Rl.Z_q = 0.0;
+    Rl.kappa = Zl; Rl.nsteps = 0;
+    Rl.cut_p = __ldcg(&rpl->cut); Rl.cut_q = -CUDART_INF_F;
+    Rl.next_child = -1;
+    Rl.status = badl ? (__ldcg(&rpl->bad) == ROW_TIMEOUT ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE) : 0;
+    Rl.bonus = -1; Rl.bonus_margin = 0.f;
+    Rl.w_in = trav ? thr_c : 1.0;
+    Rl.thr = thr_c;
+    if (P.prune && (ord >> 31) && (double)u < thr_c) atomicMin(P.best + b, (ord >> 8) & 255u);
+}
+
+// A node of weight 0 (Traversal), finished by the warp that found it out: its record, weight 0 for its children
+// (childless ones are finished on the spot), and the arrival of all of them.  W: the node's scalars.
+__device__ __noinline__ void dead_node(const VParams &P, const RowPart *part, const NodeScalars &W)
+{
+    const int lane = threadIdx.x & 31;
+    const int a = W.a, b = W.b;
+    NodeRec *rec = P.rec + (long long)b * P.N;
+    if (lane == 0) {
+        NodeRec &Rc = rec[a];
+        Rc.O_p = (double)W.O_p; Rc.Z_p = W.Z_p; Rc.O_q = (double)W.O_q; Rc.Z_q = W.Z_q;
+        Rc.kappa = W.Z_p; Rc.nsteps = 0;
+        Rc.cut_p = W.cut_p; Rc.cut_q = W.cut_q;
+        Rc.next_child = -1;
+        Rc.status = 0;
+        Rc.bonus = -1; Rc.bonus_margin = 0.f;
+        Rc.thr = 0.0;
+    }
+    unsigned narr = 1u;
+    for (int j = 0; j < W.kc; ++j) {
+        const int c = W.child[j];
+        if ((W.leaf_mask >> j) & 1u) { leaf_record(P, part, b, c, 0.0, 0u, 0.f); ++narr; continue; }
+        if (lane == 0) {
+            rec[c].w_in = 0.0;
+            *(volatile unsigned long long *)(P.w_pub + (long long)b * P.N + c) = 0ull;
+        }
+    }
+    __syncwarp();
+    arrive_sequence(P, b, narr);
 }
 
 // bounded poll of a published weight; W_PENDING when the limit ran out
@@ -269,15 +324,22 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             }
 
             // ---- the scalars block of this item -----------------------------------------------------------------
+            // A node whose weight is known to be 0 never reaches the consumers: its scalars go to the producer's
+            // own block, and the first CTA's producer finishes it at once (behind the consumers' current item it
+            // would hold up its sequence's arrivals for nothing).  Every CTA takes the same decision.
+            const bool own_block = trav && hint_dead && t >= P.B && t < total;
             const int sbuf = sidx & 1;
-            if (sidx >= 2) {
-                int w = 1;
-                if (lane == 0) w = mbar_wait(&S.sempty[sbuf], (uint32_t)(((sidx >> 1) - 1) & 1)) ? 1 : 0;
-                w = __shfl_sync(0xffffffffu, w, 0);
-                if (!w) S.poison = 1;
-            }
-            ++sidx;
-            NodeScalars &N = S.sc[sbuf];
+            auto claim_block = [&]() {
+                if (sidx >= 2) {
+                    int w = 1;
+                    if (lane == 0) w = mbar_wait(&S.sempty[sbuf], (uint32_t)(((sidx >> 1) - 1) & 1)) ? 1 : 0;
+                    w = __shfl_sync(0xffffffffu, w, 0);
+                    if (!w) S.poison = 1;
+                }
+                ++sidx;
+            };
+            if (!own_block) claim_block();
+            NodeScalars &N = own_block ? S.scd : S.sc[sbuf];
             int kind, a = 0, b = 0;
             bool hq = false;
             if (t >= total + P.B || *(volatile int *)&S.poison) {
@@ -410,6 +472,20 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             }
             if (lane == 0) N.kind = kind;
             __syncwarp();
+            if (own_block) {
+                if (kind == ITEM_DEAD && N.err == 0 && N.kc <= KMAX) {
+                    if (rank == 0) dead_node(P, TP.part, N);
+                    continue;
+                }
+                // (a faulty node after all: it goes to the consumers like any other item)
+                claim_block();
+                {
+                    const int *src = reinterpret_cast<const int *>(&S.scd);
+                    int *dst = reinterpret_cast<int *>(&S.sc[sbuf]);
+                    for (int i = lane; i < (int)(sizeof(NodeScalars) / 4); i += 32) dst[i] = src[i];
+                }
+                __syncwarp();
+            }
             if (lane == 0) mbar_arrive(&S.sfull[sbuf]);
             if (kind != ITEM_NODE && kind != ITEM_FINISH) continue;
 
@@ -485,24 +561,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
             // a childless child is finished here, by the scribe warp: its record; its arrival is made with the node's
             unsigned narr = 1u;
             auto finish_leaf = [&](int c, double thr_c, int j = -1) {
-                if (lane == 0) {
-                    NodeRec &Rl = P.rec[(long long)b * P.N + c];
-                    const RowPart *rpl = TP.part + ((long long)b * P.N + c) * 2;
-                    const double Zl = __ldcg(&rpl->S);
-                    const int Ol = __ldcg(&rpl->O);
-                    const bool badl = __ldcg(&rpl->bad) != 0 || !(Ol > ROWPART_EMPTY) || !(Zl > 0.0) || !(Zl < CUDART_INF);
-                    Rl.O_p = (double)Ol; Rl.Z_p = Zl; Rl.O_q = 0.0; Rl.Z_q = 0.0;
-                    Rl.kappa = Zl; Rl.nsteps = 0;
-                    Rl.cut_p = __ldcg(&rpl->cut); Rl.cut_q = -CUDART_INF_F;
-                    Rl.next_child = -1;
-                    Rl.status = badl ? (__ldcg(&rpl->bad) == ROW_TIMEOUT ? SPEC_DEV_TIMEOUT : SPEC_DEV_NONFINITE) : 0;
-                    Rl.bonus = -1; Rl.bonus_margin = 0.f;
-                    Rl.w_in = trav ? thr_c : 1.0;
-                    Rl.thr = thr_c;
-                    // accepted if reached: nothing that comes after it in the traversal order matters any more
-                    if (P.prune && j >= 0 && (W.cord[j] >> 31) && (double)W.cu[j] < thr_c)
-                        atomicMin(P.best + b, (W.cord[j] >> 8) & 255u);
-                }
+                leaf_record(P, TP.part, b, c, thr_c, j >= 0 ? W.cord[j] : 0u, j >= 0 ? W.cu[j] : 0.f);
                 ++narr;
             };
 
