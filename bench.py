@@ -38,7 +38,7 @@ STAT_KERNEL = {False: "stream::spec_row_partial_kernel (row statistics: the one 
                True: "trunc::spec_row_trunc_kernel (+ rowstat::spec_row_stat_kernel for the rows it leaves over)"}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of that kernel from the ncu captures summarised
 # under profiles/ (cold L2).  Workloads without a capture: null.
-TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_798_912 + 760_320}
+TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_799_168 + 626_432}
 
 
 def parse_args():
