@@ -266,3 +266,23 @@ def test_traversal_weight_one_with_a_vanishing_residual():
     batch = make_batch(w, seed=106, device="cuda")
     check_batch(batch, "traversal", full=True)
     check_batch(batch, "specinfer", full=True)
+
+
+def test_traversal_skipping_does_not_change_the_outcome():
+    """Without per-node diagnostics the Traversal call skips subtrees that come wholly after a node already
+    known to be accepted, and nodes below a weight of 0.  Outcome and residual must be those of the call
+    that evaluates every node (diagnostics on), on trees wide and deep enough for both kinds of skipping."""
+    skipped_something = 0
+    for seed in range(10):
+        w = small("skip", 6000, "bf16", 4, 2, 4, 6, sigma=0.6)
+        batch = make_batch(w, seed=seed, device="cuda")
+        plain = gpu_verify(batch, "traversal", residual=True)
+        full = gpu_verify(batch, "traversal", residual=True, node_thr=True, node_w_in=True, margin=True)
+        for name in ("accepted_node", "accept_len", "bonus_token", "out_tokens", "status"):
+            assert torch.equal(getattr(plain, name), getattr(full, name)), (seed, name)
+        assert torch.equal(plain.residual, full.residual), seed
+        # the accepted node is rarely the last one in traversal order: then there was something to skip
+        N = w.N
+        skipped_something += int((full.accepted_node != 0).sum().item())
+        assert (full.node_thr[:, 0] == 1.0).all() and full.node_thr.shape == (w.B, N)
+    assert skipped_something > 0
