@@ -143,6 +143,22 @@ int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, in
                               void *stream);
 
 /*
+ * Top-down verification with one of the other OTLP solvers the paper defines (Appendix B; composed as
+ * Section 3.2 "OT-based algorithms" says: at a node the solver puts out one token; the walk moves to the
+ * first child, in list order, that carries it, and stops when no child does -- that token is the
+ * correction token).  solver: 0 = NSS (Algorithm 1: the token is drawn from p, the drafts are ignored),
+ * 1 = NaiveTree (Algorithm 2: the first child is tested with min(1, p/q), otherwise a draw from
+ * norm((p - q)+)), 2 = SpecTr K-SEQ (Algorithm 3: division factor rho* by bisection, every child
+ * tested with min(1, p / (rho q)), otherwise a draw from its residual).  A child's test uses its entry
+ * of u_accept, a draw at node a the entry u_bonus[a].  Same inputs, workspace, stream and status rules
+ * as spec_verify_specinfer; of SpecOut only accepted_node, accept_len, out_tokens, bonus_token and
+ * status are written, and the optional outputs must be NULL (SPEC_ERR_UNSUPPORTED otherwise, and for
+ * N > 128).  solver outside 0..2: SPEC_ERR_PARAM.
+ */
+int32_t spec_verify_otlp(const SpecIn *in, const SpecOut *out, int32_t solver, void *ws, int64_t ws_bytes,
+                         void *stream);
+
+/*
  * SpecInfer verification for callers that cannot allocate device memory.  The paper has no
  * counterpart to this entry point: it exists for hosts of this library that are handed their
  * device buffers by someone else and may not call cudaMalloc themselves -- a plugin running inside

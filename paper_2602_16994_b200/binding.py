@@ -27,7 +27,8 @@ ERRORS = {0: "SPEC_OK", -1: "SPEC_ERR_NULL", -2: "SPEC_ERR_SHAPE", -3: "SPEC_ERR
 EXPORTS = ("spec_workspace_bytes", "spec_tree_probs", "spec_verify_specinfer", "spec_verify_traversal",
            "spec_sample_bonus", "spec_query_plan", "spec_host_staging_bytes", "spec_verify_host",
            "spec_verify_specinfer_static", "spec_kernel_launches", "spec_analysis_workspace_bytes",
-           "spec_tree_analysis", "spec_latency_model", "spec_test_hooks", "spec_row_statistics")
+           "spec_tree_analysis", "spec_latency_model", "spec_test_hooks", "spec_row_statistics",
+           "spec_verify_otlp")
 
 
 class SpecIn(C.Structure):
@@ -99,6 +100,8 @@ def load_library(path: str = LIB_PATH):
     lib.spec_latency_model.restype = C.c_int32
     lib.spec_latency_model.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
+    lib.spec_verify_otlp.restype = C.c_int32
+    lib.spec_verify_otlp.argtypes = [C.POINTER(SpecIn), C.POINTER(SpecOut), C.c_int32, C.c_void_p, C.c_int64, C.c_void_p]
     lib.spec_row_statistics.restype = C.c_int32
     lib.spec_row_statistics.argtypes = [C.POINTER(SpecIn), C.c_void_p, C.c_int64, C.c_void_p]
     lib.spec_test_hooks.restype = C.c_int32
@@ -264,6 +267,28 @@ def verify_specinfer(target_logits, draft_logits, parent, token, u_accept, u_bon
                  temperature_per_seq)
     return _verify("spec_verify_specinfer", m, outputs, workspace, stream, residual=residual,
                    node_thr=node_thr, features=features, margin=margin)
+
+
+OTLP_SOLVERS = {"nss": 0, "naive": 1, "spectr": 2}
+
+
+def verify_otlp(solver, target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature=1.0, top_k=0,
+                top_p=1.0, temperature_per_seq=None, outputs=None, workspace=None, stream=None):
+    """Top-down verification with NSS, NaiveTree or SpecTr (``solver``: "nss", "naive", "spectr")."""
+    lib = load_library()
+    if not torch.cuda.is_available():
+        raise RuntimeError("no CUDA device: the verification path has no CPU fallback")
+    spec_in, keep = _marshal(target_logits, draft_logits, parent, token, u_accept, u_bonus, temperature, top_k, top_p,
+                             temperature_per_seq)
+    device = target_logits.device
+    if outputs is None:
+        outputs = alloc_outputs(spec_in.B, spec_in.N, spec_in.V, device)
+    ws = workspace or _ws_for(device)
+    ptr, size = ws.get(workspace_bytes(spec_in))
+    so = outputs.as_struct()
+    _check(lib.spec_verify_otlp(C.byref(spec_in), C.byref(so), OTLP_SOLVERS[solver], ptr, size, _stream_ptr(stream)),
+           "spec_verify_otlp")
+    return outputs
 
 
 def verify_specinfer_static(target_logits, draft_logits, parent, token, u_accept, u_bonus, outputs,

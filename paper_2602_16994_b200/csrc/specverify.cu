@@ -374,10 +374,10 @@ int launch_rowstat(const SpecIn *in, const void *zp, const void *zq, const int *
 }
 
 // SpecInfer without diagnostic outputs: row statistics of every row, then one walk per sequence
-template <int DT, int NW, int MINB>
+template <int DT, int NW, int MINB, bool OT = false>
 int launch_walk(const VPlan &pl, WParams &wp, cudaStream_t st)
 {
-    auto kernel = spec_walk_kernel<DT, NW, MINB>;
+    auto kernel = spec_walk_kernel<DT, NW, MINB, OT>;
     int rc = prepare_kernel(kernel, pl.C, pl.smem);
     if (rc) return rc;
     const int threads = (NW + 1) * 32;
@@ -458,7 +458,7 @@ int row_statistics(const SpecIn *in, const SpecOut *out, unsigned char *w, const
 }
 
 int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const WsLayout &L, const VPlan &pl,
-                bool trunc, bool parts, cudaStream_t st)
+                bool trunc, bool parts, cudaStream_t st, int solver = -1)
 {
     int rc = row_statistics(in, out, w, L, trunc, parts, st);
     if (rc) return rc;
@@ -473,6 +473,12 @@ int verify_walk(const SpecIn *in, const SpecOut *out, unsigned char *w, const Ws
     wp.parent = in->parent; wp.token = in->token; wp.T = in->temperature; wp.T_seq = in->temperature_per_seq;
     wp.part = part; wp.u_accept = in->u_accept; wp.u_bonus = in->u_bonus; wp.out = *out;
     const bool bf = in->logits_dtype == SPEC_BF16;
+    if (solver >= 0) {
+        // the walk with another OTLP solver (Algorithms 1-3): its own instantiation, two CTAs per SM
+        wp.solver = solver;
+        if (pl.NW == 7) return bf ? launch_walk<SPEC_BF16, 7, 2, true>(pl, wp, st) : launch_walk<SPEC_F32, 7, 2, true>(pl, wp, st);
+        return bf ? launch_walk<SPEC_BF16, 15, 1, true>(pl, wp, st) : launch_walk<SPEC_F32, 15, 1, true>(pl, wp, st);
+    }
     if (pl.NW == 7 && pl.whole_sm) return bf ? launch_walk<SPEC_BF16, 7, 1>(pl, wp, st) : launch_walk<SPEC_F32, 7, 1>(pl, wp, st);
     if (pl.NW == 7) return bf ? launch_walk<SPEC_BF16, 7, 2>(pl, wp, st) : launch_walk<SPEC_F32, 7, 2>(pl, wp, st);
     return bf ? launch_walk<SPEC_BF16, 15, 1>(pl, wp, st) : launch_walk<SPEC_F32, 15, 1>(pl, wp, st);
@@ -688,6 +694,23 @@ int32_t spec_verify_specinfer(const SpecIn *in, const SpecOut *out, void *ws, in
 int32_t spec_verify_traversal(const SpecIn *in, const SpecOut *out, void *ws, int64_t ws_bytes, void *stream)
 {
     return verify_common(in, out, ws, ws_bytes, stream, MODE_TRAVERSAL);
+}
+
+int32_t spec_verify_otlp(const SpecIn *in, const SpecOut *out, int32_t solver, void *ws, int64_t ws_bytes, void *stream)
+{
+    int rc = check_in(in, true);
+    if (rc) return rc;
+    if (!out || !out->accepted_node || !out->accept_len || !out->out_tokens || !out->bonus_token || !out->status)
+        return SPEC_ERR_NULL;
+    if (solver < 0 || solver > 2) return SPEC_ERR_PARAM;
+    if (out->residual || out->node_thr || out->node_w_in || out->margin || out->node_features || in->N > NWALK)
+        return SPEC_ERR_UNSUPPORTED;
+    const bool trunc = (in->top_k > 0 && in->top_k < in->V) || in->top_p < 1.f;
+    const WsLayout L = ws_layout(in);
+    if (!ws || ((uintptr_t)ws & 255) || ws_bytes < L.total) return SPEC_ERR_WORKSPACE;
+    VPlan wpl;
+    if (!make_vplan(in->V, in->logits_dtype, &wpl, (int)sizeof(WHdr), false)) return SPEC_ERR_UNSUPPORTED;
+    return verify_walk(in, out, (unsigned char *)ws, L, wpl, trunc, true, (cudaStream_t)stream, solver);
 }
 
 int32_t spec_verify_specinfer_static(const SpecIn *in, const SpecOut *out, void *stream)

@@ -535,6 +535,44 @@ __device__ __forceinline__ double step_sweep(float4 *es, int nsm, int tid, Resid
     return d;
 }
 
+// SpecTr's residual (Algorithm 3) in place, in the units of the resident e_p: u <- (u - gm min(u ir, e_q r))+
+// with ir = 1 / rho, r = Z_p / Z_q, gm = gamma, for the thread's fp32 tail tokens and for the entry of the
+// warp's exact list that falls to its lane.  Returns the thread's sum of the new u.
+template <int NW>
+__device__ __forceinline__ double spectr_sweep(float4 *es, int nsm, int tid, Resident &R, WarpList &L, int nl, double gm,
+                                               double ir, double r)
+{
+    constexpr int NCONS = NW * 32;
+    const float gf = (float)gm, irf = (float)ir, rf = (float)r;
+    float tot = 0.f;
+    for (int i = 0; i < nsm; ++i) {
+        float u[8], q[8];
+        float4 *d = es + (size_t)(i * 4) * NCONS + tid;
+        load_e8(d, NCONS, u);
+        load_e8(d + 2 * NCONS, NCONS, q);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { u[k] = fmaxf(u[k] - gf * fminf(u[k] * irf, q[k] * rf), 0.f); tot += u[k]; }
+        d[0] = make_float4(u[0], u[1], u[2], u[3]);
+        d[NCONS] = make_float4(u[4], u[5], u[6], u[7]);
+    }
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            R.p[j][k] = fmaxf(R.p[j][k] - gf * fminf(R.p[j][k] * irf, R.q[j][k] * rf), 0.f);
+            tot += R.p[j][k];
+        }
+    }
+    double d = (double)tot;
+    const int lane = tid & 31;
+    if (lane < nl) {
+        const double v = fmax(L.ep[lane] - gm * fmin(L.ep[lane] * ir, L.eq[lane] * r), 0.0);
+        L.ep[lane] = v;
+        d += v;
+    }
+    return d;
+}
+
 // A read-only sweep over the thread's share of the resident node for the offline analysis: f.tail(e_p, e_q,
 // a0, a1) on every fp32 token (two running sums), f.exact(...) in fp64 on the entry of the warp's exact
 // list that falls to the lane.  Listed tokens are zero in the fp32 arrays; every f maps (0, 0) to nothing.

@@ -20,6 +20,7 @@
 // bit-identical totals to all of them), so control flow agrees across the cluster without barriers.
 // The thread that finds the bonus token writes all outputs of the sequence.
 #pragma once
+#include "analysis.cuh"
 #include "stream.cuh"
 #include "verify.cuh"
 
@@ -38,6 +39,7 @@ struct WParams {
     const RowPart *part;      // [B*N*2][NSL]
     const float *u_accept, *u_bonus;
     SpecOut out;
+    int solver;               // OT instantiation: 0 NSS (Algorithm 1), 1 NaiveTree (Algorithm 2), 2 SpecTr (Algorithm 3)
 };
 
 struct __align__(16) WHdr {
@@ -64,7 +66,10 @@ struct RowSum {
 };
 
 // MINB: CTAs per SM the register budget is set for (1: up to 255 registers per thread, no spills)
-template <int DT, int NW, int MINB>
+// OT: the walk with one of the other OTLP solvers of Appendix B instead of SpecInfer (Section 3.2: move to the
+// child whose token the solver put out, stop when the output is no child's token).  Every draw is then
+// made known to the whole cluster (one more exchange), because the walk may go on from it.
+template <int DT, int NW, int MINB, bool OT = false>
 __global__ void __launch_bounds__((NW + 1) * 32, MINB) spec_walk_kernel(const WParams P)
 {
     constexpr int NCONS = NW * 32;
@@ -258,6 +263,174 @@ __global__ void __launch_bounds__((NW + 1) * 32, MINB) spec_walk_kernel(const WP
                 rp.Z = S.t_Z[2 * a]; rp.O = S.t_O[2 * a]; rp.cut = S.t_cut[2 * a];
                 rq = rp;
                 if (hq) { rq.Z = S.t_Z[2 * a + 1]; rq.O = S.t_O[2 * a + 1]; rq.cut = S.t_cut[2 * a + 1]; }
+                if (OT) {
+                    // ================= Algorithms 1-3 at node a =================================================
+                    const int solver = P.solver;
+                    const bool use_q = hq && solver != 0;            // Algorithm 1 ignores the drafts
+                    // Algorithm 2 tests the first child only; Algorithm 3 with one child has rho = 1 and is the same
+                    const bool one_test = use_q && (solver == 1 || kc == 1);
+                    int acc = -1;
+                    if (one_test) {
+                        const double ep = S.t_cp[c_first], eq = S.t_cq[c_first];
+                        const bool zero = !(ep > 0.0), one = !zero && !(eq > 0.0);
+                        if (!zero && (one || (double)S.t_u[c_first] * eq * rp.Z < ep * rq.Z)) acc = c_first;
+                    }
+                    if (acc < 0) {
+                        if (kc > 1) {
+                            __syncwarp();
+                            int seen = 0;
+                            for (int c0 = a + 1; c0 < P.N && seen < kc; c0 += 32) {
+                                const int c = c0 + lane;
+                                const bool is = c < P.N && S.t_parent[c] == a;
+                                const unsigned bal = __ballot_sync(0xffffffffu, is);
+                                if (is) {
+                                    const int pos = seen + __popc(bal & ((1u << lane) - 1u));
+                                    W.child[pos] = c; W.cpm[pos] = S.t_cp[c]; W.cqm[pos] = S.t_cq[c]; W.cu[pos] = S.t_u[c];
+                                }
+                                seen += __popc(bal);
+                            }
+                            __syncwarp();
+                        }
+                        if (warp == 0 && lane == 0) {
+                            if (posted) { if (!mbar_wait(&S.ack, aphase)) S.poison = 1; aphase ^= 1u; }
+                            S.req_a = a; S.req_b = b; S.req_hq = use_q ? 1 : 0;
+                            mbar_arrive(&S.req);
+                            posted = true;
+                        }
+                        bool poisoned = *(volatile int *)&S.poison != 0;
+                        nr.hq = use_q; nr.cut_p = rp.cut; nr.cut_q = rq.cut; nr.O_p = rp.O; nr.O_q = rq.O;
+                        set_list_thresholds(nr, rp.Z, rq.Z);
+                        int nl;
+                        float zs_p, zs_q;
+                        pass1<DT, NW>(rc, stage, phase, poisoned, nr, es, nsm, nrg, n_slice, tid, R, L, nl, zs_p, zs_q);
+                        double Z_q = rq.Z, kappa, tot_r, Zr_q = 0.0;
+                        {
+                            const double v[2] = {warp_sum_once((double)zs_p + (lane < nl ? L.ep[lane] : 0.0)),
+                                                 warp_sum_once((double)zs_q + (lane < nl ? L.eq[lane] : 0.0))};
+                            double tot[2], mine[2];
+                            cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                            kappa = tot[0]; tot_r = mine[0];
+                            if (use_q && tot[1] > 0.0) { Z_q = tot[1]; Zr_q = mine[1]; }
+                        }
+                        if (*(volatile int *)&S.poison) status = SPEC_DEV_TIMEOUT;
+                        else if (!(kappa > 0.0)) status = SPEC_DEV_NONFINITE;
+                        const double invZq = use_q ? __drcp_rn(Z_q) : 0.0;
+                        bool is_q = false;
+                        if (!status && one_test) {
+                            // the first child was rejected: Y ~ norm((p - q)+), one step of the recursion of verify.cuh
+                            const double g = __ddiv_rn(Z_q, kappa);
+                            const double v[1] = {warp_sum_once(step_sweep<NW>(es, nsm, tid, R, L, nl, g))};
+                            double tot[1], mine[1];
+                            cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                            if (*(volatile int *)&S.poison) status = SPEC_DEV_TIMEOUT;
+                            else if (tot[0] * invZq > RESIDUAL_FLOOR) { kappa = tot[0]; tot_r = mine[0]; }
+                            else { is_q = true; kappa = Z_q; tot_r = Zr_q; }      // S = 0: p = q, drawn from q's row
+                        } else if (!status && use_q) {
+                            // ---- Algorithm 3 with k >= 2 children: the division factor by bisection (Appendix B) ----
+                            const double ip = __drcp_rn(kappa), kd = (double)kc;
+                            auto sweep2 = [&](auto f, double &t0, double &t1) {
+                                double o0, o1;
+                                reduce_sweep<NW>(es, nsm, tid, R, L, nl, f, o0, o1);
+                                const double v[2] = {warp_sum_once(o0), warp_sum_once(o1)};
+                                double tot[2], mine[2];
+                                cluster_exchange<NW, 2>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                                t0 = tot[0]; t1 = tot[1];
+                            };
+                            double lo = 1.0, hi = kd, dummy, beta;
+                            for (int it = 0; it < 40; ++it) {
+                                const double mid = 0.5 * (lo + hi), ipr = ip / mid;
+                                sweep2(FnBeta{(float)ipr, (float)invZq, ipr, invZq}, beta, dummy);
+                                const double f = (1.0 - pow(1.0 - beta, kd)) - mid * beta;
+                                if (f > 0.0) lo = mid; else hi = mid;
+                            }
+                            const double rho = 0.5 * (lo + hi);
+                            {
+                                const double ipr = ip / rho;
+                                sweep2(FnBeta{(float)ipr, (float)invZq, ipr, invZq}, beta, dummy);
+                            }
+                            const double pacc = 1.0 - pow(1.0 - beta, kd);
+                            const double gamma = beta > 0.0 ? pacc / beta : 0.0;
+                            // the children in list order, each against min(1, p(x) / (rho q(x)))
+                            const double ux = lane < kc ? W.cpm[lane] : 0.0, eqx = lane < kc ? W.cqm[lane] : 0.0;
+                            for (int j = 0; j < kc; ++j) {
+                                const double Pp = __shfl_sync(0xffffffffu, ux, j) * ip;
+                                const double Pq = __shfl_sync(0xffffffffu, eqx, j) * invZq;
+                                double thr;
+                                if (!(Pp > 0.0)) thr = 0.0;
+                                else if (!(Pq > 0.0)) thr = 1.0;
+                                else thr = fmin(1.0, (Pp / Pq) / rho);
+                                if ((double)W.cu[j] < thr) {
+                                    // the solver's output is the child's TOKEN: the walk moves to the first child,
+                                    // in list order, that carries it (duplicates stay separate nodes)
+                                    const int y = S.t_token[W.child[j]];
+                                    for (int i = 0; i <= j && acc < 0; ++i)
+                                        if (S.t_token[W.child[i]] == y) acc = W.child[i];
+                                    break;
+                                }
+                            }
+                            if (acc < 0) {
+                                // all rejected: Y ~ norm((p - min(p / rho, q) gamma)+); p itself where that is empty
+                                const double ib = beta < 1.0 ? 1.0 / (1.0 - beta) : 0.0;
+                                double sres, sacc;
+                                sweep2(FnSpecTrRes{(float)ip, (float)invZq, (float)(1.0 / rho), (float)gamma, (float)ib, (float)kd,
+                                                   ip, invZq, 1.0 / rho, gamma, ib, kd}, sres, sacc);
+                                if (sres > 0.0) {
+                                    const double v[1] = {warp_sum_once(
+                                        spectr_sweep<NW>(es, nsm, tid, R, L, nl, gamma, 1.0 / rho, kappa * invZq))};
+                                    double tot[1], mine[1];
+                                    cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                                    kappa = tot[0]; tot_r = mine[0];
+                                    if (!(kappa > 0.0)) status = SPEC_DEV_NONFINITE;
+                                }
+                            }
+                            if (*(volatile int *)&S.poison) status = SPEC_DEV_TIMEOUT;
+                        }
+                        if (!status && acc < 0) {
+                            // ---- the draw, and its token made known to every warp of the cluster ---------------------
+                            const double E_tot = warp_sum_once(lane < C ? tot_r : 0.0);
+                            const double target = (double)S.t_ub[a] * E_tot;
+                            double tau;
+                            const int owner = pick_lane(lane < C ? tot_r : 0.0, target, tau);
+                            double say = 0.0;             // token + 1 from the one thread that found it; -role on a failure
+                            if (owner < 0) {
+                                status = SPEC_DEV_NONFINITE;
+                            } else {
+                                if (owner == (int)rank) {
+                                    const BonusFind bf = bonus_search<NW>(S.wtile, &S.cbar, cph, &S.poison, es, nsm, tid, R, L, nl,
+                                                                          is_q, tau);
+                                    if (bf.role == 1) say = (double)(tok0 + bf.token) + 1.0;
+                                    else if (bf.role >= 2) say = -(double)bf.role;
+                                }
+                                const double v[1] = {warp_sum_once(say)};
+                                double tot[1], mine[1];
+                                cluster_exchange<NW, 1>(xchg, S.xbar, xn, C, rank, warp, lane, &S.poison, v, tot, mine);
+                                if (*(volatile int *)&S.poison || tot[0] == -3.0) status = SPEC_DEV_TIMEOUT;
+                                else if (!(tot[0] >= 1.0)) status = SPEC_DEV_NONFINITE;
+                                else {
+                                    const int y = (int)(tot[0] - 1.0);
+                                    // the first child, in list order, that carries the token
+                                    if (hq) {
+                                        if (kc == 1) { if (S.t_token[c_first] == y) acc = c_first; }
+                                        else
+                                            for (int j = 0; j < kc && acc < 0; ++j)
+                                                if (S.t_token[W.child[j]] == y) acc = W.child[j];
+                                    }
+                                    if (acc < 0) {
+                                        done = true;
+                                        bonus = y;
+                                        if (rank == 0 && warp == 0 && lane == 0) writer = true;
+                                    }
+                                }
+                            }
+                        }
+                        if (status) {
+                            done = true;
+                            if (rank == 0 && warp == 0 && lane == 0) { writer = true; cur = -1; len = -1; }
+                        }
+                    }
+                    if (acc >= 0 && !done) { cur = acc; ++len; }
+                    continue;
+                }
                 // ---- first child: needs no residual -------------------------------------------------------------------
                 int acc = -1;
                 int j0 = 0;
