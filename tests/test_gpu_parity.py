@@ -286,3 +286,21 @@ def test_traversal_skipping_does_not_change_the_outcome():
         skipped_something += int((full.accepted_node != 0).sum().item())
         assert (full.node_thr[:, 0] == 1.0).all() and full.node_thr.shape == (w.B, N)
     assert skipped_something > 0
+
+
+TREE_SHAPES = [
+    Workload("s_k8_root", 6, 3000, "bf16", 8, 0, 3, 0.6),        # N = 25: a wide root
+    Workload("s_k2_deep", 6, 2000, "f32", 2, 3, 6, 0.4),          # N = 16: deep branches
+    Workload("s_k5_d1", 6, 5000, "bf16", 5, 1, 6, 0.5),           # N = 32: the largest tree with a post-order table
+    Workload("s_k6_d1", 4, 4000, "bf16", 6, 1, 6, 0.5),           # N = 38: no table, nothing skipped by rank
+]
+
+
+@pytest.mark.parametrize("w", TREE_SHAPES, ids=lambda w: w.name)
+def test_traversal_on_wide_and_deep_trees(w):
+    """Traversal's hand-out hints (weight 0 at an ancestor, subtree after a known acceptance) on trees of other
+    shapes than the configs', at and beyond the size limit of the post-order table."""
+    total = Tally()
+    for seed in range(100, 108):
+        total.add(check_batch(make_batch(w, seed=seed, device="cuda"), "traversal", full=(seed % 4 == 0)))
+    assert total.near_margin_mismatches <= 1, vars(total)
