@@ -39,6 +39,9 @@ STAT_KERNEL = {False: "stream::spec_row_partial_kernel (row statistics: the one 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of that kernel from the ncu captures summarised
 # under profiles/ (cold L2).  Workloads without a capture: null.
 TRAFFIC_BYTES = {"cfg2_llama3_b8": 69_799_168 + 626_432}
+# the same counters summed over the kernels of a whole call, captured in one pass without cache flushes between
+# the kernels (profiles/per_config.md): the second kernel of a call finds most of its rows in L2
+TRAFFIC_CALL_BYTES = {"cfg2_llama3_b8": {"specinfer": 70_810_000 + 90_000, "traversal": 70_810_000 + 9_200_000}}
 
 
 def parse_args():
@@ -433,7 +436,8 @@ def run_ours(args):
                      "frac_of_8TBs_nominal": achieved / 8000.0,
                      "traffic": None if trunc else TRAFFIC_BYTES.get(w.name),
                      "algorithmic_bytes_per_launch": bytes_per_call,
-                     "whole_call_frac": {a: per_algo[a]["gbs"] / peak for a in w.algorithms}},
+                     "whole_call_frac": {a: per_algo[a]["gbs"] / peak for a in w.algorithms},
+                     "whole_call_traffic": None if trunc else TRAFFIC_CALL_BYTES.get(w.name)},
         "l2_warm_us": l2_warm,
         "clocks": clocks, "gpu_launches": gpu_launches,
         "status_ok": status_ok,
