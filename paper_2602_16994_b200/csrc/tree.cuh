@@ -371,9 +371,12 @@ __global__ void __launch_bounds__((NW + 1) * 32, NW <= 7 ? 2 : 1) spec_tree_kern
                 } else {
                     a = acc;
                     const NodeRec *rc = P.rec + (long long)b * P.N + a;
+                    // (all coefficient slots are fetched, in the same round of loads as the step count: only the first
+                    // nsteps are read by the consumers)
+                    const double gj = lane < KMAX ? __ldcg(TP.gseq + ((long long)b * P.N + a) * KMAX + lane) : 0.0;
                     const int nsteps = __ldcg(&rc->nsteps);
                     hq = nsteps != 0;
-                    if (lane < KMAX && lane < nsteps) N.cpm[lane] = __ldcg(TP.gseq + ((long long)b * P.N + a) * KMAX + lane);
+                    if (lane < KMAX) N.cpm[lane] = gj;
                     if (lane == 0) {
                         N.Z_p = __ldcg(&rc->Z_p); N.Z_q = __ldcg(&rc->Z_q);
                         N.O_p = (int)__ldcg(&rc->O_p); N.O_q = (int)__ldcg(&rc->O_q);
